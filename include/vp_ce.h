@@ -1,0 +1,117 @@
+/*
+ * vp_ce.h -- C ABI of the fused vocabulary projection + cross-entropy library (sm_100a).
+ *
+ * The operation (paper section 3.2, Eq. 2; Appendix C, Algorithm 3): logits Y = H * W^T are
+ * formed one vocabulary shard ("strip") at a time; every strip is folded into a per-token
+ * running state S = (m, z, y_t) and dropped, so the tokens x vocabulary matrix never exists.
+ * After all shards the negative log-likelihood of a token is m + log z - y_t.  Backward
+ * replays the same meetings from the saved normaliser lse = m + log z, forms the softmax
+ * residual of one strip at a time and contracts it into the input and weight gradients.
+ * On one device the ring of Algorithm 3 is a loop over shards: token chunk c (global index
+ * chunk_index_base + local chunk) meets shard q_i = (c - i) mod P at step i = 0..P-1, with
+ * P = ceil(V / block_v).
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller unless a parameter is
+ *     explicitly called "host".  Inputs are never written.  The library allocates and
+ *     frees no device memory in these calls; scratch memory is the caller's `workspace`.
+ *   - Layouts (row-major, no padding):
+ *       H      [T, d]  bfloat16      hidden states
+ *       W      [V, d]  bfloat16      projection weight (logits = H * W^T)
+ *       labels [T]     int32         target ids in [0, V) or ignore_index
+ *       loss, lse, dloss [T] float32
+ *       dH     [T, d]  bfloat16      dW [V, d] float32
+ *   - H, W, dH, dW and workspace must be 16-byte aligned; d must be a multiple of 8;
+ *     block_v must be a multiple of 256 and T_chunk a multiple of 128 (tile shapes).
+ *   - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on that stream
+ *     and do not synchronise with the host.  The return value reports host-detectable
+ *     errors only; conditions found on the device (a label outside [0, V) that is not
+ *     ignore_index; a bounded wait inside a kernel that ran out) set a status word in the
+ *     workspace, read back with vp_ce_device_status.
+ *   - A token whose label equals ignore_index has loss 0 and a zero gradient row; its lse
+ *     is still computed.  A label outside [0, V) is treated the same way and flagged.
+ */
+#ifndef VP_CE_H_
+#define VP_CE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int vpce_status;
+#define VPCE_OK                  0
+#define VPCE_INVALID_ARG         1  /* null pointer, non-positive size                        */
+#define VPCE_UNSUPPORTED         2  /* alignment or divisibility rule above not met           */
+#define VPCE_WORKSPACE_TOO_SMALL 3
+#define VPCE_CUDA_ERROR          4  /* a CUDA runtime/driver call or a launch failed          */
+
+/* Bits of the device status word (vp_ce_device_status). */
+#define VPCE_DEV_LABEL_OUT_OF_RANGE 1
+#define VPCE_DEV_WAIT_EXPIRED       2
+
+/*
+ * Bytes of workspace needed by vp_ce_forward / vp_ce_backward for a given token chunk,
+ * hidden width and shard width.  Depends on neither V nor T (Eq. 1 of section 3.2: the live
+ * logit memory is O(N V / P) = O(T_chunk * block_v)).  Pure host arithmetic; returns 0 for
+ * arguments that the other calls would reject.
+ */
+size_t vp_ce_workspace_bytes(int64_t T_chunk, int64_t d, int64_t block_v);
+
+/*
+ * Forward (Algorithm 3 with Fold = Eq. 2, output line "m + log z - y").
+ * Writes lse[n] for every token and loss[n] = lse[n] - y[n, labels[n]] (0 if ignored).
+ * T_chunk: tokens per internal chunk (the paper's per-rank batch N); chunk c covers tokens
+ * [c*T_chunk, min(T, (c+1)*T_chunk)).  chunk_index_base: global index of this call's first
+ * chunk (rotation of the shard order when a long stream is cut into several calls).
+ * The workspace contents are undefined on entry and on return except for the status word,
+ * which this call clears first.
+ */
+vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels,
+                          int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                          float* loss, float* lse,
+                          int64_t T_chunk, int64_t chunk_index_base,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Backward (Appendix C: replay the meetings from the saved per-token normaliser).
+ * lse: the forward's output.  dloss: per-token upstream gradient of loss[n], or NULL for
+ * the masked mean (1 / n_valid on valid tokens, n_valid counted from labels; 0 valid tokens
+ * give zero gradients).  dH is overwritten.  dW is overwritten when accumulate_dW == 0 and
+ * added to otherwise (fp32 accumulation across calls of a streamed context).
+ */
+vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse,
+                           const float* dloss, void* dH, float* dW,
+                           int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                           int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Masked mean of the per-token loss (not part of the paper's operator, which outputs
+ * per-token values; this is the reduction the benchmark's metric is stated on).
+ * mean_out[0] = sum of loss over valid tokens / n_valid (0 when n_valid == 0);
+ * n_valid_out[0] = n_valid.  Both are device pointers.  Deterministic (fixed order).
+ */
+vpce_status vp_ce_mean_loss(const float* loss, const int32_t* labels, int64_t T, int64_t V,
+                            int32_t ignore_index, float* mean_out, int32_t* n_valid_out, void* stream);
+
+/*
+ * Copies the device status word of `workspace` to host_out[0] (HOST pointer) and
+ * synchronises `stream`.  0 means no device-side condition was seen since the last
+ * vp_ce_forward / vp_ce_backward call on this workspace began.
+ */
+vpce_status vp_ce_device_status(const void* workspace, int32_t* host_out, void* stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char* vp_ce_status_string(vpce_status s);
+
+/* Number of kernels the library launched on behalf of the caller since the process
+ * started (monotonic, host-side counter; used by the benchmark's launch accounting). */
+int64_t vp_ce_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VP_CE_H_ */

@@ -1,0 +1,17 @@
+"""B200-native fused vocabulary projection + cross-entropy (single-device Ring-DTP, paper §3.2 / App. C).
+
+The package is a thin binding over the C-ABI library ``libvpce.so`` (hand-written sm_100a
+kernels).  There is no CPU or PyTorch fallback: every call raises if the library is missing.
+"""
+from .binding import (  # noqa: F401
+    VpceError,
+    library_path,
+    load_library,
+    vp_ce_backward,
+    vp_ce_device_status,
+    vp_ce_forward,
+    vp_ce_launch_count,
+    vp_ce_mean_loss,
+    vp_ce_status_string,
+    vp_ce_workspace_bytes,
+)

@@ -1,0 +1,145 @@
+"""ctypes binding of libvpce.so: argument marshalling only, same names as the C entry points.
+
+Tensors are torch CUDA tensors (torch supplies device memory and streams); the binding
+checks dtype/shape/contiguity, passes raw device pointers and the current stream, and turns
+non-zero status codes into ``VpceError``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+_LIB: Optional[ctypes.CDLL] = None
+_LIB_NAME = "libvpce.so"
+
+
+class VpceError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"vp_ce status {code}: {msg}")
+        self.code = code
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), _LIB_NAME)
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the in-tree CUDA library; raises if it has not been built (no fallback exists)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(
+            f"{path} is missing: build it with `python -m paper_2609_14306_b200.build` "
+            "(or __graft_entry__.build()); this package has no CPU fallback")
+    lib = ctypes.CDLL(path)
+    i64, i32, vp, sz = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t
+    lib.vp_ce_workspace_bytes.restype = sz
+    lib.vp_ce_workspace_bytes.argtypes = [i64, i64, i64]
+    lib.vp_ce_forward.restype = ctypes.c_int
+    lib.vp_ce_forward.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, i64, i64, vp, sz, vp]
+    lib.vp_ce_backward.restype = ctypes.c_int
+    lib.vp_ce_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, i64, i64,
+                                   ctypes.c_int, vp, sz, vp]
+    lib.vp_ce_mean_loss.restype = ctypes.c_int
+    lib.vp_ce_mean_loss.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
+    lib.vp_ce_device_status.restype = ctypes.c_int
+    lib.vp_ce_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+    lib.vp_ce_status_string.restype = ctypes.c_char_p
+    lib.vp_ce_status_string.argtypes = [ctypes.c_int]
+    lib.vp_ce_launch_count.restype = i64
+    lib.vp_ce_launch_count.argtypes = []
+    _LIB = lib
+    return lib
+
+
+def _check(code: int) -> None:
+    if code != 0:
+        raise VpceError(code, vp_ce_status_string(code))
+
+
+def vp_ce_status_string(code: int) -> str:
+    return load_library().vp_ce_status_string(int(code)).decode()
+
+
+def vp_ce_launch_count() -> int:
+    return int(load_library().vp_ce_launch_count())
+
+
+def vp_ce_workspace_bytes(T_chunk: int, d: int, block_v: int) -> int:
+    return int(load_library().vp_ce_workspace_bytes(int(T_chunk), int(d), int(block_v)))
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _ptr(t, dtype, name: str, numel: Optional[int] = None) -> int:
+    import torch
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if numel is not None and t.numel() != numel:
+        raise ValueError(f"{name} has {t.numel()} elements, expected {numel}")
+    return int(t.data_ptr())
+
+
+def _shapes(H, W) -> Tuple[int, int, int]:
+    if H.dim() != 2 or W.dim() != 2 or H.shape[1] != W.shape[1]:
+        raise ValueError("H must be [T, d] and W [V, d]")
+    return int(H.shape[0]), int(H.shape[1]), int(W.shape[0])
+
+
+def vp_ce_forward(H, W, labels, block_v: int, ignore_index: int, loss, lse, T_chunk: int,
+                  chunk_index_base: int, workspace, stream=None) -> None:
+    """loss[n], lse[n] for every token (Algorithm 3); see include/vp_ce.h for the contract."""
+    import torch
+    lib = load_library()
+    T, d, V = _shapes(H, W)
+    _check(lib.vp_ce_forward(
+        _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
+        T, d, V, int(block_v), int(ignore_index),
+        _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
+        int(T_chunk), int(chunk_index_base),
+        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+
+
+def vp_ce_backward(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index: int, T_chunk: int,
+                   chunk_index_base: int, accumulate_dW: bool, workspace, stream=None) -> None:
+    """dH (bf16, overwritten) and dW (fp32, overwritten or accumulated); dloss may be None."""
+    import torch
+    lib = load_library()
+    T, d, V = _shapes(H, W)
+    _check(lib.vp_ce_backward(
+        _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
+        _ptr(lse, torch.float32, "lse", T),
+        None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
+        _ptr(dH, torch.bfloat16, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
+        T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
+        1 if accumulate_dW else 0,
+        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+
+
+def vp_ce_mean_loss(loss, labels, V: int, ignore_index: int, mean_out, n_valid_out, stream=None) -> None:
+    import torch
+    lib = load_library()
+    T = loss.numel()
+    _check(lib.vp_ce_mean_loss(
+        _ptr(loss, torch.float32, "loss"), _ptr(labels, torch.int32, "labels", T), T, int(V), int(ignore_index),
+        _ptr(mean_out, torch.float32, "mean_out", 1), _ptr(n_valid_out, torch.int32, "n_valid_out", 1),
+        _stream_ptr(stream)))
+
+
+def vp_ce_device_status(workspace, stream=None) -> int:
+    import torch
+    lib = load_library()
+    out = ctypes.c_int32(-1)
+    _check(lib.vp_ce_device_status(_ptr(workspace, torch.uint8, "workspace"), ctypes.byref(out), _stream_ptr(stream)))
+    return int(out.value)

@@ -1,0 +1,895 @@
+// Fused vocabulary projection + cross-entropy for sm_100a (B200).
+//
+// One warp-specialised, persistent tcgen05 GEMM kernel is instantiated with four epilogues:
+//   FOLD   strip Y = H_c W_q^T  -> per-tile partial (max, sum-exp) + target logit   (Eq. 2)
+//   RESID  the same strip       -> G = dloss (exp(Y - lse) - onehot) as bf16       (App. C)
+//   DH     dH_c += G W_q        (contract over the shard's vocabulary)
+//   DW     dW_q += G^T H_c      (contract over the chunk's tokens)
+// Operands reach shared memory by TMA (128-byte swizzle), accumulators live in tensor
+// memory (two buffers, so the epilogue of tile i overlaps the MMAs of tile i+1), and the
+// logit strip never reaches global memory.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
+// warps 2..5 = epilogue (one thread per accumulator row).
+//
+// Every wait on an mbarrier is bounded: when it runs out the CTA records
+// VPCE_DEV_WAIT_EXPIRED in the workspace status word, all roles leave their loops, pending
+// copies and MMAs are drained (bounded again), TMEM is freed and the kernel returns.
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstdio>
+#include <mutex>
+
+#include "vp_ce.h"
+
+namespace {
+
+constexpr int BM = 128;          // accumulator rows per tile (TMEM lanes)
+constexpr int BK = 64;           // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
+constexpr int BN_VOCAB = 256;    // vocabulary columns per strip tile
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARP0 = 2;
+constexpr int SMEM_BUDGET = 200 * 1024;    // operand stages
+constexpr int SMEM_EXTRA = 2048;           // barriers + alignment slack
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
+
+enum Epilogue { EPI_FOLD = 0, EPI_RESID = 1, EPI_DH = 2, EPI_DW = 3 };
+
+struct GemmParams {
+    int m_tiles, n_tiles, num_kb;
+    int a_mn0, a_k0, b_mn0, b_k0;          // TMA coordinate bases (elements)
+    int rows_valid;                        // valid accumulator rows overall (M bound)
+    int cols_valid;                        // valid accumulator columns overall (N bound)
+    // FOLD / RESID
+    int v_lo;                              // first vocabulary id of the shard
+    const int32_t* labels;                 // chunk base
+    const float* lse;                      // chunk base
+    const float* dloss;                    // chunk base or null
+    const float* inv_n_valid;              // scalar used when dloss == null
+    int ignore_index;
+    int V;
+    float* pm;                             // [n_tile][part_ld] partial max
+    float* pz;                             // [n_tile][part_ld] partial sum-exp
+    float* ylab;                           // [part_ld] target logit
+    int part_ld;
+    __nv_bfloat16* G;                      // [T_chunk][g_ld]
+    int g_ld;
+    // DH
+    float* acc;                            // [T_chunk][acc_ld] fp32 running dH of the chunk
+    int acc_ld;
+    __nv_bfloat16* dH;                     // chunk base, leading dimension out_ld
+    int first, last;
+    // DW
+    float* dW;                             // shard base (row v_lo), leading dimension out_ld
+    int accumulate;
+    int out_ld;
+    int* status;
+};
+
+// ------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor (sm_100 format), 128-byte swizzle.
+//   K-major operand : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (SBO); LBO unused.
+//   MN-major operand: 64 K-rows of 64 MN elements (128 B) per box; boxes of successive
+//                     64-element MN chunks LBO bytes apart; 8-K-row groups 1024 B apart (SBO).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;                      // descriptor version of sm_100
+    d |= 2ull << 61;                      // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = 128, N = bn.
+__host__ __device__ constexpr uint32_t make_idesc(int bn, bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn) << 15) |
+           (static_cast<uint32_t>(b_mn) << 16) | (static_cast<uint32_t>(bn >> 3) << 17) |
+           (static_cast<uint32_t>(BM >> 4) << 24);
+}
+
+template <int BN> struct StageCfg {
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
+    static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// ------------------------------------------------------------------------------------ epilogues
+// Each epilogue thread owns accumulator row `row` (0..127) of the tile; `tmem_row` is the
+// TMEM address of that thread's lane quadrant at the accumulator's first column.
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float NEG_INF = -__builtin_huge_valf();
+
+__device__ __forceinline__ void epilogue_fold(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+    const int grow = mt * BM + row;                             // row within the chunk
+    const bool row_ok = grow < p.rows_valid;
+    const int label = row_ok ? p.labels[grow] : -1;
+    const int lrel = label - (p.v_lo + nt * BN_VOCAB);          // target column relative to the tile
+    float m = NEG_INF, z = 0.f, yl = 0.f;
+    bool hit = false;
+#pragma unroll 1
+    for (int c = 0; c < BN_VOCAB / 32; ++c) {
+        float v[32];
+        __syncwarp();
+        tmem_ld32(tmem_row + c * 32, v);
+        tmem_ld_wait();
+        const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);     // valid columns left in the shard
+        if (nvalid < 32) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (j >= nvalid) v[j] = NEG_INF;
+        }
+        if (static_cast<unsigned>(lrel - c * 32) < 32u) {
+            const int jj = lrel - c * 32;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (j == jj) yl = v[j];
+            hit = true;
+        }
+        float cmax = v[0];
+#pragma unroll
+        for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
+        const float m_new = fmaxf(m, cmax);
+        const float mL = (m_new == NEG_INF) ? 0.f : m_new * LOG2E;
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) s += ex2f(fmaf(v[j], LOG2E, -mL));
+        z = z * ex2f(fmaf(m, LOG2E, -mL)) + s;                         // m = -inf gives factor 0
+        m = m_new;
+    }
+    if (row_ok) {
+        p.pm[static_cast<size_t>(nt) * p.part_ld + grow] = m;
+        p.pz[static_cast<size_t>(nt) * p.part_ld + grow] = z;
+        if (hit) p.ylab[grow] = yl;                                    // exactly one tile owns the target
+    }
+}
+
+__device__ __forceinline__ void epilogue_resid(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+    const int grow = mt * BM + row;
+    const bool row_ok = grow < p.rows_valid;
+    int label = row_ok ? p.labels[grow] : p.ignore_index;
+    const bool valid = row_ok && label != p.ignore_index && static_cast<unsigned>(label) < static_cast<unsigned>(p.V);
+    float dl = 0.f, lseL = 0.f;
+    if (valid) dl = p.dloss ? p.dloss[grow] : *p.inv_n_valid;
+    if (row_ok) lseL = p.lse[grow] * LOG2E;
+    const int lrel = valid ? label - (p.v_lo + nt * BN_VOCAB) : -1;
+    __nv_bfloat16* grow_ptr = p.G + static_cast<size_t>(grow) * p.g_ld + nt * BN_VOCAB;
+#pragma unroll 1
+    for (int c = 0; c < BN_VOCAB / 32; ++c) {
+        float v[32];
+        __syncwarp();
+        tmem_ld32(tmem_row + c * 32, v);
+        tmem_ld_wait();
+        const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);
+        const int jj = lrel - c * 32;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            float g = dl * ex2f(fmaf(v[j], LOG2E, -lseL));
+            if (j == jj) g -= dl;
+            v[j] = (j < nvalid) ? g : 0.f;
+        }
+        uint4* dst = reinterpret_cast<uint4*>(grow_ptr + c * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint4 o;
+            o.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
+            o.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+            o.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+            o.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+            dst[q] = o;                                                // rows >= rows_valid get zeros
+        }
+    }
+}
+
+template <int BN>
+__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+    const int grow = mt * BM + row;
+    const bool row_ok = grow < p.rows_valid;
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+        float v[32];
+        __syncwarp();
+        tmem_ld32(tmem_row + c * 32, v);
+        tmem_ld_wait();
+        const int col0 = nt * BN + c * 32;
+        if (row_ok) {
+        float* arow = p.acc + static_cast<size_t>(grow) * p.acc_ld + col0;
+        __nv_bfloat16* orow = p.dH + static_cast<size_t>(grow) * p.out_ld + col0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {                                  // 8 columns per step
+            if (col0 + 8 * q >= p.cols_valid) break;                   // d is a multiple of 8
+            float* x = v + 8 * q;
+            if (!p.first) {
+                const float4 a0 = *reinterpret_cast<const float4*>(arow + 8 * q);
+                const float4 a1 = *reinterpret_cast<const float4*>(arow + 8 * q + 4);
+                x[0] += a0.x; x[1] += a0.y; x[2] += a0.z; x[3] += a0.w;
+                x[4] += a1.x; x[5] += a1.y; x[6] += a1.z; x[7] += a1.w;
+            }
+            if (p.last) {
+                uint4 o;
+                o.x = pack_bf16x2(x[0], x[1]); o.y = pack_bf16x2(x[2], x[3]);
+                o.z = pack_bf16x2(x[4], x[5]); o.w = pack_bf16x2(x[6], x[7]);
+                *reinterpret_cast<uint4*>(orow + 8 * q) = o;
+            } else {
+                *reinterpret_cast<float4*>(arow + 8 * q) = make_float4(x[0], x[1], x[2], x[3]);
+                *reinterpret_cast<float4*>(arow + 8 * q + 4) = make_float4(x[4], x[5], x[6], x[7]);
+            }
+        }
+        }
+    }
+}
+
+template <int BN>
+__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+    const int grow = mt * BM + row;                                    // vocabulary row within the shard
+    const bool row_ok = grow < p.rows_valid;
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+        float v[32];
+        __syncwarp();
+        tmem_ld32(tmem_row + c * 32, v);
+        tmem_ld_wait();
+        const int col0 = nt * BN + c * 32;
+        if (row_ok) {
+        float* orow = p.dW + static_cast<size_t>(grow) * p.out_ld + col0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {                                  // 4 columns per step
+            if (col0 + 4 * q >= p.cols_valid) break;
+            float4 x = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            if (p.accumulate) {
+                const float4 a = *reinterpret_cast<const float4*>(orow + 4 * q);
+                x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
+            }
+            *reinterpret_cast<float4*>(orow + 4 * q) = x;
+        }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ the GEMM kernel
+template <int BN, bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+    using Cfg = StageCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr uint32_t TMEM_COLS = (BN > 128) ? 512u : (BN > 64 ? 256u : 128u);
+    constexpr uint32_t ACC_STRIDE = TMEM_COLS / 2;
+    constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;                      // swizzle atoms need 1024-byte alignment
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t bars = base + STAGES * Cfg::STAGE_BYTES;            // 8-byte barriers after the stages
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            long issued = 0;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
+                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+                    if (A_MN) {
+#pragma unroll
+                        for (int j = 0; j < BM / 64; ++j)
+                            tma_load_2d(sa + j * (BK * 128), &tmA, full_bar(stage), p.a_mn0 + mt * BM + 64 * j, p.a_k0 + kb * BK);
+                    } else {
+                        tma_load_2d(sa, &tmA, full_bar(stage), p.a_k0 + kb * BK, p.a_mn0 + mt * BM);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j)
+                            tma_load_2d(sb + j * (BK * 128), &tmB, full_bar(stage), p.b_mn0 + nt * BN + 64 * j, p.b_k0 + kb * BK);
+                    } else {
+                        tma_load_2d(sb, &tmB, full_bar(stage), p.b_k0 + kb * BK, p.b_mn0 + nt * BN);
+                    }
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok || *abort_flag) {
+                // Give-up path: let this CTA's copies in flight land before shared memory is released.
+                const long back = issued < STAGES ? issued : STAGES;
+                int s = stage; uint32_t ph = phase;
+                for (long i = 0; i < back; ++i) {
+                    if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
+                    unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+                const int ab = it & 1;
+                const uint32_t aphase = (it >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+                    const uint64_t adesc = A_MN ? make_smem_desc(sa, BK * 128, 1024) : make_smem_desc(sa, 16, 1024);
+                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, BK * 128, 1024) : make_smem_desc(sb, 16, 1024);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // K-major: 16 elements = 32 B along the swizzled row; MN-major: 16 K-rows = 2048 B
+                        const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
+                        const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
+                        umma_f16(tmem_d, adesc + aoff, bdesc + boff, IDESC, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));                      // frees the stage once these MMAs retire
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(tfull_bar(ab));
+            }
+            if (!ok || *abort_flag) {
+                umma_commit(drain_bar);                                 // wait for MMAs still in flight
+                unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int quad = warp & 3;                                     // TMEM lane quadrant this warp may read
+        const int row = quad * 32 + lane;
+        int it = 0; bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+            const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+            const int ab = it & 1;
+            const uint32_t aphase = (it >> 1) & 1u;
+            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
+            if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
+            else if (EPI == EPI_RESID) epilogue_resid(p, mt, nt, row, tmem_row);
+            else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row);
+            else epilogue_dw<BN>(p, mt, nt, row, tmem_row);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(ab));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, VPCE_DEV_WAIT_EXPIRED);
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------ small kernels
+// Folds the per-tile partial states of one strip into the running per-token state (Eq. 2
+// applied to two states: m = max(m1, m2), z = z1 e^{m1-m} + z2 e^{m2-m}), in tile order so the
+// result does not depend on which CTA produced which tile.  On the last step it also emits
+// lse = m + log z and loss = lse - y_t (Algorithm 3, output line).
+__global__ void vpce_merge_kernel(const float* __restrict__ pm, const float* __restrict__ pz, int part_ld, int n_tiles,
+                                  float* __restrict__ sm, float* __restrict__ sz, const float* __restrict__ ylab,
+                                  int rows, int first, int last, const int32_t* __restrict__ labels, int ignore_index,
+                                  int V, float* __restrict__ lse, float* __restrict__ loss, int* status) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= rows) return;
+    float m = first ? NEG_INF : sm[n];
+    float z = first ? 0.f : sz[n];
+    for (int t = 0; t < n_tiles; ++t) {
+        const float m2 = pm[static_cast<size_t>(t) * part_ld + n];
+        const float z2 = pz[static_cast<size_t>(t) * part_ld + n];
+        const float mn = fmaxf(m, m2);
+        z = z * ex2f((m - mn) * LOG2E) + z2 * ex2f((m2 - mn) * LOG2E);   // m = -inf contributes 0
+        m = mn;
+    }
+    if (!last) { sm[n] = m; sz[n] = z; return; }
+    const float l = m + logf(z);
+    lse[n] = l;
+    const int t = labels[n];
+    float out = 0.f;
+    if (t != ignore_index) {
+        if (static_cast<unsigned>(t) < static_cast<unsigned>(V)) out = l - ylab[n];
+        else atomicOr(status, VPCE_DEV_LABEL_OUT_OF_RANGE);
+    }
+    loss[n] = out;
+}
+
+// One block: counts valid labels (fixed order) and stores 1 / n_valid (0 when there is none).
+__global__ void vpce_count_valid_kernel(const int32_t* __restrict__ labels, long T, int V, int ignore_index,
+                                        float* inv_n_valid, int* n_valid_out, int* status) {
+    __shared__ int part[1024];
+    int c = 0, bad = 0;
+    for (long i = threadIdx.x; i < T; i += blockDim.x) {
+        const int t = labels[i];
+        if (t != ignore_index) {
+            if (static_cast<unsigned>(t) < static_cast<unsigned>(V)) ++c; else bad = 1;
+        }
+    }
+    if (bad && status) atomicOr(status, VPCE_DEV_LABEL_OUT_OF_RANGE);
+    part[threadIdx.x] = c;
+    __syncthreads();
+    for (int s = blockDim.x / 2; s > 0; s >>= 1) {
+        if (threadIdx.x < s) part[threadIdx.x] += part[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (inv_n_valid) *inv_n_valid = part[0] > 0 ? 1.0f / static_cast<float>(part[0]) : 0.f;
+        if (n_valid_out) *n_valid_out = part[0];
+    }
+}
+
+// One block: masked mean of the per-token loss, double accumulation in a fixed order.
+__global__ void vpce_mean_loss_kernel(const float* __restrict__ loss, const int32_t* __restrict__ labels, long T, int V,
+                                      int ignore_index, float* mean_out, int* n_valid_out) {
+    __shared__ double sums[1024];
+    __shared__ int cnts[1024];
+    double s = 0.0; int c = 0;
+    for (long i = threadIdx.x; i < T; i += blockDim.x) {
+        const int t = labels[i];
+        if (t != ignore_index && static_cast<unsigned>(t) < static_cast<unsigned>(V)) { s += loss[i]; ++c; }
+    }
+    sums[threadIdx.x] = s; cnts[threadIdx.x] = c;
+    __syncthreads();
+    for (int k = blockDim.x / 2; k > 0; k >>= 1) {
+        if (threadIdx.x < k) { sums[threadIdx.x] += sums[threadIdx.x + k]; cnts[threadIdx.x] += cnts[threadIdx.x + k]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        *mean_out = cnts[0] > 0 ? static_cast<float>(sums[0] / cnts[0]) : 0.f;
+        *n_valid_out = cnts[0];
+    }
+}
+
+__global__ void vpce_clear_status_kernel(int* status) { if (threadIdx.x < 8) status[threadIdx.x] = 0; }
+
+// ------------------------------------------------------------------------------------ host side
+std::atomic<long long> g_launches{0};
+
+struct WsLayout {
+    size_t status, scalars, sm, sz, ylab, pm, pz, G, acc, total;
+};
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool ws_layout(int64_t T_chunk, int64_t d, int64_t block_v, WsLayout* L) {
+    if (T_chunk <= 0 || d <= 0 || block_v <= 0) return false;
+    if (T_chunk % BM || block_v % BN_VOCAB || d % 8) return false;
+    if (T_chunk > (1 << 24) || block_v > (1 << 24) || d > (1 << 20)) return false;
+    const size_t nt = static_cast<size_t>(block_v / BN_VOCAB);
+    size_t off = 0;
+    L->status = off;  off += 256;
+    L->scalars = off; off += 256;
+    L->sm = off;      off = align_up(off + 4 * T_chunk, 1024);
+    L->sz = off;      off = align_up(off + 4 * T_chunk, 1024);
+    L->ylab = off;    off = align_up(off + 4 * T_chunk, 1024);
+    L->pm = off;      off = align_up(off + 4 * T_chunk * nt, 1024);
+    L->pz = off;      off = align_up(off + 4 * T_chunk * nt, 1024);
+    L->G = off;       off = align_up(off + 2 * static_cast<size_t>(T_chunk) * block_v, 1024);
+    L->acc = off;     off = align_up(off + 4 * static_cast<size_t>(T_chunk) * d, 1024);
+    L->total = off;
+    return true;
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    });
+    return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix: dim0 = cols (contiguous), 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld_elems, uint32_t box_cols,
+              uint32_t box_rows) {
+    auto enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld_elems * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int num_sms() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+template <int BN, bool A_MN, bool B_MN, int EPI>
+cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+    using Cfg = StageCfg<BN>;
+    auto kern = vpce_gemm_kernel<BN, A_MN, B_MN, EPI>;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const int tiles = p.m_tiles * p.n_tiles;
+    if (tiles <= 0 || p.num_kb <= 0) return cudaSuccess;
+    const int grid = tiles < num_sms() ? tiles : num_sms();
+    kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmA, tmB, p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+// Output-column tile for the two gradient GEMMs: the widest of {256, 192, 128, 64} that wastes
+// the fewest padded columns of d.
+int pick_bn(int64_t d) {
+    const int cands[4] = {256, 192, 128, 64};
+    int best = 256; int64_t best_pad = -1;
+    for (int c : cands) {
+        const int64_t pad = (d + c - 1) / c * c;
+        if (best_pad < 0 || pad < best_pad) { best = c; best_pad = pad; }
+    }
+    return best;
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+cudaError_t launch_grad(int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+    switch (bn) {
+        case 256: return launch_gemm<256, A_MN, B_MN, EPI>(tmA, tmB, p, st);
+        case 192: return launch_gemm<192, A_MN, B_MN, EPI>(tmA, tmB, p, st);
+        case 128: return launch_gemm<128, A_MN, B_MN, EPI>(tmA, tmB, p, st);
+        default:  return launch_gemm<64, A_MN, B_MN, EPI>(tmA, tmB, p, st);
+    }
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+vpce_status check_common(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
+                         int64_t block_v, int64_t T_chunk, int64_t chunk_index_base, const void* ws, size_t ws_bytes,
+                         WsLayout* L) {
+    if (!H || !W || !labels || !ws) return VPCE_INVALID_ARG;
+    if (T <= 0 || d <= 0 || V <= 0 || block_v <= 0 || T_chunk <= 0 || chunk_index_base < 0) return VPCE_INVALID_ARG;
+    if (!aligned16(H) || !aligned16(W) || !aligned16(ws)) return VPCE_UNSUPPORTED;
+    if (T >= (1ll << 31) || V >= (1ll << 31)) return VPCE_UNSUPPORTED;
+    if (!ws_layout(T_chunk, d, block_v, L)) return VPCE_UNSUPPORTED;
+    if (ws_bytes < L->total) return VPCE_WORKSPACE_TOO_SMALL;
+    return VPCE_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------ C ABI
+extern "C" {
+
+size_t vp_ce_workspace_bytes(int64_t T_chunk, int64_t d, int64_t block_v) {
+    WsLayout L;
+    return ws_layout(T_chunk, d, block_v, &L) ? L.total : 0;
+}
+
+const char* vp_ce_status_string(vpce_status s) {
+    switch (s) {
+        case VPCE_OK: return "ok";
+        case VPCE_INVALID_ARG: return "invalid argument (null pointer or non-positive size)";
+        case VPCE_UNSUPPORTED: return "unsupported (alignment, d % 8, block_v % 256 or T_chunk % 128)";
+        case VPCE_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case VPCE_CUDA_ERROR: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+int64_t vp_ce_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
+                          int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
+                          int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream) {
+    WsLayout L;
+    if (!loss || !lse) return VPCE_INVALID_ARG;
+    vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
+    if (s != VPCE_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws + L.status);
+    float* sm = reinterpret_cast<float*>(ws + L.sm);
+    float* sz = reinterpret_cast<float*>(ws + L.sz);
+    float* ylab = reinterpret_cast<float*>(ws + L.ylab);
+    float* pm = reinterpret_cast<float*>(ws + L.pm);
+    float* pz = reinterpret_cast<float*>(ws + L.pz);
+
+    CUtensorMap tmH, tmW;
+    if (!make_map(&tmH, H, T, d, d, BK, BM) || !make_map(&tmW, W, V, d, d, BK, BN_VOCAB)) return VPCE_CUDA_ERROR;
+
+    vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+
+    const int64_t P = (V + block_v - 1) / block_v;
+    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
+    const int num_kb = static_cast<int>((d + BK - 1) / BK);
+    for (int64_t c = 0; c < n_chunks; ++c) {
+        const int64_t tok0 = c * T_chunk;
+        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
+        const int64_t cg = chunk_index_base + c;
+        for (int64_t i = 0; i < P; ++i) {
+            const int64_t q = ((cg - i) % P + P) % P;                  // Algorithm 3: q = (r - i) mod P
+            const int64_t v_lo = q * block_v;
+            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
+            GemmParams p{};
+            p.m_tiles = (rows + BM - 1) / BM;
+            p.n_tiles = (cols + BN_VOCAB - 1) / BN_VOCAB;
+            p.num_kb = num_kb;
+            p.a_mn0 = static_cast<int>(tok0); p.a_k0 = 0;
+            p.b_mn0 = static_cast<int>(v_lo); p.b_k0 = 0;
+            p.rows_valid = rows; p.cols_valid = cols;
+            p.v_lo = static_cast<int>(v_lo);
+            p.labels = labels + tok0;
+            p.ignore_index = ignore_index; p.V = static_cast<int>(V);
+            p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
+            p.status = status;
+            if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
+                                                                  rows, i == 0, i == P - 1, labels + tok0, ignore_index,
+                                                                  static_cast<int>(V), lse + tok0, loss + tok0, status);
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return VPCE_CUDA_ERROR;
+        }
+    }
+    return VPCE_OK;
+}
+
+vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse, const float* dloss,
+                           void* dH, float* dW, int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                           int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    WsLayout L;
+    if (!lse || !dH || !dW) return VPCE_INVALID_ARG;
+    vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
+    if (s != VPCE_OK) return s;
+    if (!aligned16(dH) || !aligned16(dW)) return VPCE_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(ws + L.status);
+    float* inv_n = reinterpret_cast<float*>(ws + L.scalars);
+    __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.G);
+    float* acc = reinterpret_cast<float*>(ws + L.acc);
+
+    CUtensorMap tmH_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmH_mn;
+    if (!make_map(&tmH_k, H, T, d, d, BK, BM) || !make_map(&tmW_k, W, V, d, d, BK, BN_VOCAB) ||
+        !make_map(&tmG_k, G, T_chunk, block_v, block_v, BK, BM) || !make_map(&tmW_mn, W, V, d, d, 64, BK) ||
+        !make_map(&tmG_mn, G, T_chunk, block_v, block_v, 64, BK) || !make_map(&tmH_mn, H, T, d, d, 64, BK))
+        return VPCE_CUDA_ERROR;
+
+    vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!dloss) {
+        vpce_count_valid_kernel<<<1, 1024, 0, st>>>(labels, T, static_cast<int>(V), ignore_index, inv_n, nullptr, status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+
+    const int bn = pick_bn(d);
+    const int64_t P = (V + block_v - 1) / block_v;
+    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
+    for (int64_t c = 0; c < n_chunks; ++c) {
+        const int64_t tok0 = c * T_chunk;
+        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
+        const int64_t cg = chunk_index_base + c;
+        for (int64_t i = 0; i < P; ++i) {
+            const int64_t q = ((cg - i) % P + P) % P;
+            const int64_t v_lo = q * block_v;
+            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
+            const int strip_tiles_n = (cols + BN_VOCAB - 1) / BN_VOCAB;
+            // (1) recompute the strip and form the residual G (bf16) in the workspace
+            GemmParams p{};
+            p.m_tiles = (rows + BM - 1) / BM;
+            p.n_tiles = strip_tiles_n;
+            p.num_kb = static_cast<int>((d + BK - 1) / BK);
+            p.a_mn0 = static_cast<int>(tok0); p.b_mn0 = static_cast<int>(v_lo);
+            p.rows_valid = rows; p.cols_valid = cols;
+            p.v_lo = static_cast<int>(v_lo);
+            p.labels = labels + tok0; p.lse = lse + tok0; p.dloss = dloss ? dloss + tok0 : nullptr;
+            p.inv_n_valid = inv_n; p.ignore_index = ignore_index; p.V = static_cast<int>(V);
+            p.G = G; p.g_ld = static_cast<int>(block_v);
+            p.status = status;
+            if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            const int k_cols = strip_tiles_n * BN_VOCAB;               // columns of G written by step (1)
+            const int m_rows = p.m_tiles * BM;                         // rows of G written by step (1)
+            // (2) dH_c += G W_q : M = tokens, N = d, K = shard vocabulary
+            GemmParams ph{};
+            ph.m_tiles = p.m_tiles;
+            ph.n_tiles = static_cast<int>((d + bn - 1) / bn);
+            ph.num_kb = k_cols / BK;
+            ph.a_mn0 = 0; ph.a_k0 = 0;
+            ph.b_mn0 = 0; ph.b_k0 = static_cast<int>(v_lo);
+            ph.rows_valid = rows; ph.cols_valid = static_cast<int>(d);
+            ph.acc = acc; ph.acc_ld = static_cast<int>(d);
+            ph.dH = static_cast<__nv_bfloat16*>(dH) + tok0 * d; ph.out_ld = static_cast<int>(d);
+            ph.first = (i == 0); ph.last = (i == P - 1);
+            ph.status = status;
+            if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            // (3) dW_q += G^T H_c : M = shard vocabulary, N = d, K = chunk tokens
+            GemmParams pw{};
+            pw.m_tiles = (cols + BM - 1) / BM;
+            pw.n_tiles = ph.n_tiles;
+            pw.num_kb = m_rows / BK;
+            pw.a_mn0 = 0; pw.a_k0 = 0;
+            pw.b_mn0 = 0; pw.b_k0 = static_cast<int>(tok0);
+            pw.rows_valid = cols; pw.cols_valid = static_cast<int>(d);
+            pw.dW = dW + v_lo * d; pw.out_ld = static_cast<int>(d);
+            pw.accumulate = (accumulate_dW != 0) || (c > 0);
+            pw.status = status;
+            if (launch_grad<true, true, EPI_DW>(bn, tmG_mn, tmH_mn, pw, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+        }
+    }
+    return VPCE_OK;
+}
+
+vpce_status vp_ce_mean_loss(const float* loss, const int32_t* labels, int64_t T, int64_t V, int32_t ignore_index,
+                            float* mean_out, int32_t* n_valid_out, void* stream) {
+    if (!loss || !labels || !mean_out || !n_valid_out || T <= 0 || V <= 0) return VPCE_INVALID_ARG;
+    vpce_mean_loss_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(loss, labels, T, static_cast<int>(V),
+                                                                           ignore_index, mean_out, n_valid_out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
+}
+
+vpce_status vp_ce_device_status(const void* workspace, int32_t* host_out, void* stream) {
+    if (!workspace || !host_out) return VPCE_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(host_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return VPCE_CUDA_ERROR;
+    return cudaStreamSynchronize(st) == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
+}
+
+}  // extern "C"

@@ -1,0 +1,169 @@
+"""GPU parity: the CUDA path, called through the C-ABI, against the float64 oracle on the same
+seeded inputs.  Tolerances are the benchmark's: |lse|,|loss| err <= 2e-3 per token, mean loss
+relative error <= 1e-4, dH/dW relative Frobenius error <= 1e-2."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_14306_b200 as vp
+from oracle import vpce_oracle as orc
+from synth_inputs import (IGNORE_INDEX, WORKLOADS, bf16_bits_to_f64, custom_workload, make_batch,
+                          make_dloss)
+from vpce_testlib import (TOL_GRAD, TOL_TOKEN, GpuRun, check_against_oracle, relF)
+
+pytestmark = pytest.mark.gpu
+
+
+def full_check(w, dloss=None, base=0, tag=None):
+    b = make_batch(w)
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    run = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk, base).forward().backward(dloss)
+    assert run.fwd_status == 0 and run.bwd_status == 0
+    ref = orc.forward_backward(H64, W64, b.labels, dloss, IGNORE_INDEX)
+    dl64 = orc.default_dloss(b.labels, IGNORE_INDEX) if dloss is None else dloss.astype(np.float64)
+    e = check_against_oracle(run, ref, H64, W64, b.labels, dl64, tag or w.name)
+    print(w.name, {k: f"{v:.2e}" for k, v in e.items()})
+    return run, ref, e
+
+
+def test_config1_tiny():
+    full_check(WORKLOADS["tiny"])
+
+
+def test_config2_mid():
+    full_check(WORKLOADS["mid"])
+
+
+@pytest.mark.parametrize("T,d,V,block_v,T_chunk", [
+    (300, 256, 1280, 512, 128),     # ragged token tail, ragged last shard (256 of 512)
+    (128, 64, 700, 256, 128),       # vocabulary ends inside a tile; d = one K block
+    (640, 264, 1000, 1024, 256),    # d not a multiple of 64, single shard wider than V
+    (257, 40, 300, 256, 128),       # tiny d (one partial K block), T = 2 tiles + 1 row
+    (512, 2880, 2048, 512, 256),    # d = 2880 selects the 192-column gradient tile
+    (384, 512, 5000, 1024, 384),    # T_chunk of three tiles, 5 shards, last one ragged
+])
+def test_ragged_shapes(T, d, V, block_v, T_chunk):
+    w = custom_workload(f"r{T}x{d}x{V}", T=T, d=d, V=V, block_v=block_v, T_chunk=T_chunk,
+                        w_std=1.0 / np.sqrt(d), labels="zipf", ignore_frac=0.07, seed=T + V)
+    full_check(w, base=3)
+
+
+def test_sharp_logits_make_softmax_part_visible():
+    # logit sigma ~ 4: the softmax part of the gradients is no longer negligible next to the one-hot part
+    w = custom_workload("sharp", T=512, d=256, V=4096, block_v=512, T_chunk=256, w_std=0.25,
+                        labels="uniform", ignore_frac=0.05, seed=77)
+    _, _, e = full_check(w)
+    assert e["dW_softmax_only"] < 5e-3 and e["dH_softmax_only"] < 5e-3
+
+
+def test_explicit_dloss():
+    w = WORKLOADS["tiny"]
+    full_check(w, dloss=make_dloss(w))
+
+
+def test_all_tokens_ignored():
+    w = custom_workload("allign", T=256, d=128, V=1024, block_v=512, T_chunk=128, w_std=0.1, seed=5)
+    b = make_batch(w)
+    lab = np.full(w.T, IGNORE_INDEX, dtype=np.int32)
+    run = GpuRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward()
+    lse_ref, _ = orc.dense_forward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), lab)
+    assert np.abs(run.np_lse() - lse_ref).max() <= TOL_TOKEN
+    assert not run.np_loss().any() and not run.np_dH().any() and not run.np_dW().any()
+    assert run.mean() == (0.0, 0)
+
+
+def test_zero_weight_gives_log_V():
+    w = custom_workload("w0", T=256, d=128, V=1536, block_v=512, T_chunk=128, seed=6, ignore_frac=0.1)
+    b = make_batch(w)
+    run = GpuRun(b.H_bits, np.zeros_like(b.W_bits), b.labels, w.block_v, w.T_chunk).forward().backward()
+    valid = b.labels != IGNORE_INDEX
+    assert np.abs(run.np_lse() - np.log(w.V)).max() < 1e-5
+    assert np.abs(run.np_loss()[valid] - np.log(w.V)).max() < 1e-5
+    assert not run.np_dH().any()
+
+
+def test_label_out_of_range_sets_status_and_is_ignored():
+    w = custom_workload("oor", T=256, d=128, V=1024, block_v=512, T_chunk=128, w_std=0.1, seed=8)
+    b = make_batch(w)
+    lab = b.labels.copy()
+    lab[3] = w.V + 5
+    lab[200] = -7
+    run = GpuRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward()
+    assert run.fwd_status & 1 and run.bwd_status & 1
+    lab_ok = lab.copy()
+    lab_ok[[3, 200]] = IGNORE_INDEX
+    ref = orc.forward_backward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), lab_ok)
+    assert np.abs(run.np_loss() - ref["loss"]).max() <= TOL_TOKEN
+    assert relF(run.np_dW(), ref["dW"]) <= TOL_GRAD and relF(run.np_dH(), ref["dH"]) <= TOL_GRAD
+    # a later clean call clears the flag
+    run2 = GpuRun(b.H_bits, b.W_bits, lab_ok, w.block_v, w.T_chunk).forward()
+    assert run2.fwd_status == 0
+
+
+def test_invariance_to_block_chunk_and_rotation():
+    w = custom_workload("inv", T=512, d=256, V=3072, block_v=512, T_chunk=128, w_std=0.08,
+                        labels="zipf", ignore_frac=0.05, seed=9)
+    b = make_batch(w)
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    ref = orc.forward_backward(H64, W64, b.labels)
+    outs = []
+    for block_v, T_chunk, base in [(512, 128, 0), (1024, 256, 5), (256, 512, 1), (3072, 128, 2), (4096, 384, 0)]:
+        r = GpuRun(b.H_bits, b.W_bits, b.labels, block_v, T_chunk, base).forward().backward()
+        assert np.abs(r.np_lse() - ref["lse"]).max() <= TOL_TOKEN
+        assert relF(r.np_dH(), ref["dH"]) <= TOL_GRAD and relF(r.np_dW(), ref["dW"]) <= TOL_GRAD
+        outs.append(r.np_lse())
+    # all launch configurations agree with one another far more tightly than with the tolerance
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() < 1e-4
+
+
+def test_run_to_run_bitwise_determinism():
+    w = WORKLOADS["tiny"]
+    b = make_batch(w)
+    a = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
+    c = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
+    assert torch.equal(a.lse, c.lse) and torch.equal(a.loss, c.loss)
+    assert torch.equal(a.dH.view(torch.int16), c.dH.view(torch.int16)) and torch.equal(a.dW, c.dW)
+
+
+def test_accumulate_dW_across_calls_matches_one_call():
+    # a stream cut into two calls with chunk_index_base continuing equals one call over all tokens
+    w = custom_workload("acc", T=512, d=256, V=2048, block_v=512, T_chunk=128, w_std=0.08,
+                        labels="zipf", ignore_frac=0.05, seed=10)
+    b = make_batch(w)
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    dl = orc.default_dloss(b.labels, IGNORE_INDEX)
+    ref = orc.forward_backward(H64, W64, b.labels, dl)
+    half = w.T // 2
+    Wd = None
+    dW = torch.zeros(w.V, w.d, dtype=torch.float32, device="cuda")
+    parts = []
+    for k in range(2):
+        sl = slice(k * half, (k + 1) * half)
+        r = GpuRun(b.H_bits[sl], b.W_bits, b.labels[sl], w.block_v, w.T_chunk, chunk_index_base=k * (half // w.T_chunk),
+                   W_dev=Wd, dW=dW)
+        Wd = r.W
+        r.forward().backward(dloss=dl[sl].astype(np.float32), accumulate=True)
+        parts.append(r)
+    assert relF(dW.cpu().numpy(), ref["dW"]) <= TOL_GRAD
+    assert relF(np.concatenate([p.np_dH() for p in parts]), ref["dH"]) <= TOL_GRAD
+    assert np.abs(np.concatenate([p.np_lse() for p in parts]) - ref["lse"]).max() <= TOL_TOKEN
+
+
+def test_host_side_argument_checks():
+    w = WORKLOADS["tiny"]
+    b = make_batch(w)
+    r = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(vp.VpceError) as ei:
+        vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, 0, small)
+    assert ei.value.code == 3
+    with pytest.raises(vp.VpceError) as ei:
+        vp.vp_ce_forward(r.H, r.W, r.labels, 500, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, 0, r.ws)
+    assert ei.value.code == 2
+    with pytest.raises(vp.VpceError) as ei:
+        vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, 100, 0, r.ws)
+    assert ei.value.code == 2
+    with pytest.raises(vp.VpceError) as ei:
+        vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, -1, r.ws)
+    assert ei.value.code == 1

@@ -1,0 +1,54 @@
+"""CPU-side checks of the boundary: the library builds, loads, exports every symbol the header
+declares, and its pure-host entry points behave (no kernel is launched here)."""
+import ctypes
+import os
+import re
+
+import paper_2609_14306_b200 as vp
+from paper_2609_14306_b200.build import build_library
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    names = []
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if fn.endswith(".h"):
+            text = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, fn)).read(), flags=re.S)
+            names += re.findall(r"\b(vp_ce_\w+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol():
+    build_library()
+    lib = vp.load_library()
+    names = declared_functions()
+    assert {"vp_ce_forward", "vp_ce_backward", "vp_ce_workspace_bytes", "vp_ce_mean_loss",
+            "vp_ce_device_status", "vp_ce_status_string"} <= set(names)
+    raw = ctypes.CDLL(vp.library_path())
+    for n in names:
+        assert hasattr(raw, n), n
+        assert hasattr(vp, n), f"python binding lacks {n}"
+
+
+def test_workspace_size_depends_on_neither_V_nor_T():
+    # cfg 3 and cfg 5 share (T_chunk, d, block_v), hence the workspace
+    a = vp.vp_ce_workspace_bytes(4096, 2880, 8192)
+    assert a > 0 and a == vp.vp_ce_workspace_bytes(4096, 2880, 8192)
+    g = 4096 * 8192 * 2 + 4096 * 2880 * 4
+    assert g <= a <= g + (4 << 20)          # G strip + fp32 dH accumulator + O(T_chunk) state
+    assert vp.vp_ce_workspace_bytes(8192, 7168, 8192) > a
+    # rejected shapes
+    assert vp.vp_ce_workspace_bytes(100, 2880, 8192) == 0      # T_chunk % 128
+    assert vp.vp_ce_workspace_bytes(4096, 2881, 8192) == 0     # d % 8
+    assert vp.vp_ce_workspace_bytes(4096, 2880, 8000) == 0     # block_v % 256
+    assert vp.vp_ce_workspace_bytes(0, 2880, 8192) == 0
+
+
+def test_status_strings():
+    assert vp.vp_ce_status_string(0) == "ok"
+    for c in (1, 2, 3, 4):
+        assert vp.vp_ce_status_string(c) not in ("ok", "unknown status")
+    assert vp.vp_ce_status_string(99) == "unknown status"
+    assert vp.vp_ce_launch_count() >= 0
