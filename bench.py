@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the fused vocabulary projection + cross-entropy path (forward + backward).
+
+One "step" is one pass of the whole hot path over one synthetic batch: vp_ce_forward, then
+vp_ce_backward (masked-mean upstream gradient), then vp_ce_mean_loss; for the long-context
+workload a step is the whole stream (64 calls, dW accumulated across calls).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is tokens/s with inputs resident in HBM; `e2e` is the
+same metric through vp_ce_fwd_bwd_host with pinned HOST activations (copies inside the timed
+region).  With N > 1 every rank runs an independent replica on its own batch (the path has no
+exchange step on one node: weak scaling, no collective in the data path).
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "fused vocab-proj CE fwd+bwd tokens/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+# Token chunk used by the timed launch configuration (a call argument of the library).
+BENCH_T_CHUNK = {"tiny": 128, "mid": 2048, "moe120b": 8192, "moe667b": 8192, "longctx": 8192}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 6:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample_rate(w, W_bits, H_bits, labels, budget_s=15.0):
+    """Times the float64 oracle (as it stands) on the first n tokens of the batch against the whole
+    vocabulary; n is sized from a short probe so that the timed call takes about `budget_s`."""
+    from oracle import vpce_oracle as orc
+    from synth_inputs import IGNORE_INDEX, bf16_bits_to_f64
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    W64 = bf16_bits_to_f64(W_bits)
+    probe = min(32, w.T)
+    t0 = time.perf_counter()
+    orc.forward_backward(bf16_bits_to_f64(H_bits[:probe]), W64, labels[:probe], None, IGNORE_INDEX)
+    per_tok = (time.perf_counter() - t0) / probe
+    n = int(max(probe, min(w.T, budget_s / max(per_tok, 1e-9))))
+    n = max(32, (n // 32) * 32) if w.T >= 32 else w.T
+    n = min(n, w.T)
+    t0 = time.perf_counter()
+    orc.forward_backward(bf16_bits_to_f64(H_bits[:n]), W64, labels[:n], None, IGNORE_INDEX)
+    dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": "tokens/s", "cores": int(cores), "kind": "oracle",
+            "sample": f"first {n} of {w.T} tokens of one call against the full vocabulary V={w.V}, d={w.d}: "
+                      f"float64 forward+backward by the dense definition, {dt:.1f} s wall clock"}, n, dt
+
+
+def run_reference(args, w):
+    """The reference arm: the oracle on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from synth_inputs import make_hidden, make_weights, stream_labels
+    W_bits = make_weights(w)
+    labels = stream_labels(w)[:w.T]
+    H_bits = make_hidden(w, 0)
+    steps = max(1, args.steps)
+    budget = max(2.0, min(15.0, 120.0 / (steps + args.warmup)))
+    res, n, dt = None, 0, 0.0
+    times = []
+    for i in range(args.warmup + steps):
+        res, n, dt = oracle_sample_rate(w, W_bits, H_bits, labels, budget_s=budget)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = n / (ms / 1e3)
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+           "steps": steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": w.name, "T": w.T, "d": w.d, "V": w.V, "block_v": w.block_v,
+                      "note": "float64 CPU oracle, each step a bounded token sample of the workload"},
+           "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": res["cores"], "kind": "oracle",
+                            "sample": res["sample"]},
+           "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+# --------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="moe120b")
+    ap.add_argument("--t-chunk", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile-in-timed-region", type=int, default=1)
+    args = ap.parse_args()
+
+    from synth_inputs import IGNORE_INDEX, WORKLOADS, make_hidden, make_weights, stream_labels
+    w = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import paper_2609_14306_b200 as vp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    vp.load_library()          # raises if the CUDA library is missing: there is no fallback
+
+    T_chunk = args.t_chunk or BENCH_T_CHUNK.get(w.name, w.T_chunk)
+    T_chunk = min(T_chunk, -(-w.T // 128) * 128)
+    chunks_per_call = -(-w.T // T_chunk)
+
+    # ---- inputs (host, seeded) -> device.  Each rank of a multi-GPU run draws its own batch stream.
+    W_bits = make_weights(w)
+    labels_all = stream_labels(w)
+    def bf16_dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    Wd = bf16_dev(W_bits)
+    H_host0 = make_hidden(w, 0) if rank == 0 else None
+    Hs, labs = [], []
+    for call in range(w.n_calls):
+        hb = H_host0 if (call == 0 and rank == 0) else make_hidden(
+            w if rank == 0 else dataclasses.replace(w, seed=w.seed + 1000 * rank), call)
+        Hs.append(bf16_dev(hb))
+        labs.append(torch.from_numpy(labels_all[call * w.T:(call + 1) * w.T].copy()).to(dev))
+    n_valid_total = int((labels_all != IGNORE_INDEX).sum())
+
+    torch.cuda.synchronize()
+    resident = torch.cuda.memory_allocated(dev)
+    torch.cuda.reset_peak_memory_stats(dev)
+    ws_bytes = vp.vp_ce_workspace_bytes(T_chunk, w.d, w.block_v)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    loss = [torch.empty(w.T, dtype=torch.float32, device=dev) for _ in range(w.n_calls)]
+    lse = [torch.empty(w.T, dtype=torch.float32, device=dev) for _ in range(w.n_calls)]
+    dH = [torch.empty(w.T, w.d, dtype=torch.bfloat16, device=dev) for _ in range(w.n_calls)]
+    dW = torch.empty(w.V, w.d, dtype=torch.float32, device=dev)
+    mean = torch.zeros(1, dtype=torch.float32, device=dev)
+    nval = torch.zeros(1, dtype=torch.int32, device=dev)
+    dl_stream = None
+    if w.n_calls > 1:       # streamed context: the caller supplies 1 / n_valid of the whole stream
+        dl_stream = [torch.where(l != IGNORE_INDEX, 1.0 / n_valid_total, 0.0).float() for l in labs]
+
+    def step():
+        for call in range(w.n_calls):
+            base = call * chunks_per_call
+            vp.vp_ce_forward(Hs[call], Wd, labs[call], w.block_v, IGNORE_INDEX, loss[call], lse[call], T_chunk, base, ws)
+            vp.vp_ce_backward(Hs[call], Wd, labs[call], lse[call], None if dl_stream is None else dl_stream[call],
+                              dH[call], dW, w.block_v, IGNORE_INDEX, T_chunk, base, call > 0, ws)
+            vp.vp_ce_mean_loss(loss[call], labs[call], w.V, IGNORE_INDEX, mean, nval)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert vp.vp_ce_device_status(ws) == 0, "device status word set during warm-up"
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    prof_on = bool(args.profile_in_timed_region)
+    launches0 = vp.vp_ce_launch_count()
+    vp.vp_ce_profile_enable(prof_on)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    vp.vp_ce_profile_enable(False)
+    ms_total = e0.elapsed_time(e1)
+    prof = vp.vp_ce_profile_collect() if prof_on else None
+    launches = vp.vp_ce_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    peak_extra = torch.cuda.max_memory_allocated(dev) - resident
+    mean_loss = float(mean.item())
+    status = vp.vp_ce_device_status(ws)
+
+    # ---- un-profiled control run (same K) so the event overhead of the profiled region is visible
+    ms_step_noprof = None
+    if prof_on:
+        barrier(); e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record(); barrier()
+        ms_step_noprof = e0.elapsed_time(e1) / args.steps
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e and w.n_calls == 1:
+        Hh = torch.empty(w.T, w.d, dtype=torch.bfloat16).pin_memory()
+        Hh.copy_(Hs[0].cpu())
+        lh = labs[0].cpu().pin_memory()
+        loss_h = torch.empty(w.T, dtype=torch.float32).pin_memory()
+        dH_h = torch.empty(w.T, w.d, dtype=torch.bfloat16).pin_memory()
+        H_stage = torch.empty_like(Hs[0]); lab_stage = torch.empty_like(labs[0])
+        def e2e_step():
+            vp.vp_ce_fwd_bwd_host(Hh, lh, Wd, loss_h, dH_h, dW, w.block_v, IGNORE_INDEX, T_chunk, 0, False,
+                                  H_stage, lab_stage, loss[0], lse[0], dH[0], ws)
+        for _ in range(3):
+            e2e_step()
+        barrier(); e0.record()
+        for _ in range(args.steps):
+            e2e_step()
+        e1.record(); barrier()
+        ms_e2e = e0.elapsed_time(e1)
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        ms_e2e /= args.steps
+        e2e = {"value": world * w.T_stream / (ms_e2e / 1e3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": w.T * w.d * 2 + w.T * 4, "d2h_bytes_per_step": w.T * 4 + w.T * w.d * 2,
+               "api": "vp_ce_fwd_bwd_host (pinned host H, labels in; loss, dH out; W and dW resident)",
+               "mean_loss_host": float(loss_h[lh != IGNORE_INDEX].double().mean())}
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = load_peaks()
+    tokens = w.T_stream
+    value = world * tokens / (ms_step / 1e3)
+    tflops = w.flops / (ms_step / 1e3) / 1e12
+    out = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "T": w.T, "calls_per_step": w.n_calls, "d": w.d, "V": w.V,
+                   "block_v": w.block_v, "T_chunk": T_chunk, "P": w.P, "ignored_labels": w.n_ignored,
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (W alone is %.2f GB); no flush" % (w.V * w.d * 2 / 1e9)},
+        "tflops_per_gpu": tflops,
+        "frac_of_bf16_peak": {"burst_measured": tflops / peaks["bf16_tflops"],
+                              "sustained_measured": tflops / peaks["bf16_tflops_sustained"],
+                              "nominal_2250": tflops / NOMINAL_BF16_TFLOPS, "source": peak_src},
+        "flops_per_step": w.flops,
+        "peak_bytes": {"workspace_bytes": ws_bytes, "increment_over_resident_inputs": int(peak_extra),
+                       "outputs_bytes": int(w.T_stream * 8 + w.T_stream * w.d * 2 + w.V * w.d * 4),
+                       "full_fp32_logits_bytes": w.logits_bytes_fp32,
+                       "dense_fwd_bwd_would_hold_bytes": 3 * w.logits_bytes_fp32},
+        "mean_loss": mean_loss, "device_status": status,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if ms_step_noprof is not None:
+        out["ms_per_step_without_kernel_events"] = ms_step_noprof
+    if prof:
+        # every kernel kind performs 2*T*V*d flops per step; the dominant one is the slowest in total
+        flops_kind = 2.0 * w.T_stream * w.V * w.d * args.steps
+        kinds = {}
+        for k, (ms, n) in prof.items():
+            if n:
+                kinds[k] = {"launches": n, "total_ms": ms, "avg_ms": ms / n,
+                            "tflops": flops_kind / (ms / 1e3) / 1e12}
+        dom = max(kinds, key=lambda k: kinds[k]["total_ms"])
+        ach = kinds[dom]["tflops"]
+        out["roofline"] = {"bound": "tensor", "kernel": dom, "achieved": ach, "peak": peaks["bf16_tflops"],
+                           "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                           "peak_kind": "bf16_tflops (burst), of " + peak_src,
+                           "frac_of_sustained": ach / peaks["bf16_tflops_sustained"],
+                           "flops_per_launch": flops_kind / kinds[dom]["launches"],
+                           "avg_launch_ms": kinds[dom]["avg_ms"], "traffic": None}
+        out["kernels"] = kinds
+    if e2e:
+        out["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        hb = H_host0
+        cb, _, _ = oracle_sample_rate(w, W_bits, hb, labels_all[:w.T])
+        out["cpu_baseline"] = cb
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -111,6 +111,36 @@ const char* vp_ce_status_string(vpce_status s);
  * started (monotonic, host-side counter; used by the benchmark's launch accounting). */
 int64_t vp_ce_launch_count(void);
 
+/*
+ * One whole pass (Algorithm 3 forward, then the Appendix C backward with the masked-mean
+ * upstream gradient) for callers whose activations live in HOST memory.
+ *   H_host [T, d] bf16, labels_host [T] int32          HOST, read (pinned memory makes the
+ *   loss_host [T] fp32, dH_host [T, d] bf16            HOST, written    copies asynchronous)
+ *   W [V, d] bf16, dW [V, d] fp32                      DEVICE: the weight and its gradient
+ *                                                      accumulator stay resident, as in training
+ *   H_dev, labels_dev, loss_dev, lse_dev, dH_dev       DEVICE staging buffers of the same shapes,
+ *                                                      owned by the caller; nothing is allocated here
+ * Copies H and labels to the device, runs vp_ce_forward and vp_ce_backward (dloss = NULL), copies
+ * loss and dH back, then synchronises `stream`, so the host buffers are valid on return.
+ * Errors are those of the two calls it wraps.
+ */
+vpce_status vp_ce_fwd_bwd_host(const void* H_host, const int32_t* labels_host, const void* W, float* loss_host,
+                               void* dH_host, float* dW, int64_t T, int64_t d, int64_t V, int64_t block_v,
+                               int32_t ignore_index, int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW,
+                               void* H_dev, int32_t* labels_dev, float* loss_dev, float* lse_dev, void* dH_dev,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Measurement aid (no counterpart in the paper).  While enabled, every tensor-core kernel
+ * launch is bracketed by two CUDA events on the launching stream.  vp_ce_profile_collect
+ * waits for the recorded events, adds up the elapsed milliseconds and launch counts per kernel
+ * kind into the HOST arrays ms_out[4], launches_out[4] (0 = forward strip + fold,
+ * 1 = backward strip + residual, 2 = input-gradient GEMM, 3 = weight-gradient GEMM) and
+ * forgets them.  Not thread-safe against concurrent launches from other host threads.
+ */
+void vp_ce_profile_enable(int on);
+vpce_status vp_ce_profile_collect(double* ms_out, int64_t* launches_out);
+
 #ifdef __cplusplus
 }
 #endif

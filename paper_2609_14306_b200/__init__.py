@@ -10,6 +10,10 @@ from .binding import (  # noqa: F401
     vp_ce_backward,
     vp_ce_device_status,
     vp_ce_forward,
+    vp_ce_fwd_bwd_host,
+    vp_ce_profile_collect,
+    vp_ce_profile_enable,
+    KERNEL_KINDS,
     vp_ce_launch_count,
     vp_ce_mean_loss,
     vp_ce_status_string,

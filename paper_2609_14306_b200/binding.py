@@ -51,6 +51,13 @@ def load_library() -> ctypes.CDLL:
     lib.vp_ce_status_string.argtypes = [ctypes.c_int]
     lib.vp_ce_launch_count.restype = i64
     lib.vp_ce_launch_count.argtypes = []
+    lib.vp_ce_fwd_bwd_host.restype = ctypes.c_int
+    lib.vp_ce_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, i64, i64, ctypes.c_int,
+                                       vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.vp_ce_profile_enable.restype = None
+    lib.vp_ce_profile_enable.argtypes = [ctypes.c_int]
+    lib.vp_ce_profile_collect.restype = ctypes.c_int
+    lib.vp_ce_profile_collect.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     _LIB = lib
     return lib
 
@@ -143,3 +150,47 @@ def vp_ce_device_status(workspace, stream=None) -> int:
     out = ctypes.c_int32(-1)
     _check(lib.vp_ce_device_status(_ptr(workspace, torch.uint8, "workspace"), ctypes.byref(out), _stream_ptr(stream)))
     return int(out.value)
+
+
+def _host_ptr(t, dtype, name: str, numel: int) -> int:
+    import torch
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError(f"{name} must be a CPU tensor")
+    if t.dtype != dtype or not t.is_contiguous() or t.numel() != numel:
+        raise ValueError(f"{name}: expected contiguous {dtype} with {numel} elements")
+    return int(t.data_ptr())
+
+
+def vp_ce_fwd_bwd_host(H_host, labels_host, W, loss_host, dH_host, dW, block_v: int, ignore_index: int,
+                       T_chunk: int, chunk_index_base: int, accumulate_dW: bool,
+                       H_dev, labels_dev, loss_dev, lse_dev, dH_dev, workspace, stream=None) -> None:
+    """Forward + backward with activations in host memory (copies inside the call); W/dW on device."""
+    import torch
+    lib = load_library()
+    T, d = int(H_host.shape[0]), int(H_host.shape[1])
+    V = int(W.shape[0])
+    _check(lib.vp_ce_fwd_bwd_host(
+        _host_ptr(H_host, torch.bfloat16, "H_host", T * d), _host_ptr(labels_host, torch.int32, "labels_host", T),
+        _ptr(W, torch.bfloat16, "W", V * d), _host_ptr(loss_host, torch.float32, "loss_host", T),
+        _host_ptr(dH_host, torch.bfloat16, "dH_host", T * d), _ptr(dW, torch.float32, "dW", V * d),
+        T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base), 1 if accumulate_dW else 0,
+        _ptr(H_dev, torch.bfloat16, "H_dev", T * d), _ptr(labels_dev, torch.int32, "labels_dev", T),
+        _ptr(loss_dev, torch.float32, "loss_dev", T), _ptr(lse_dev, torch.float32, "lse_dev", T),
+        _ptr(dH_dev, torch.bfloat16, "dH_dev", T * d),
+        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+
+
+KERNEL_KINDS = ("fwd_strip_fold", "bwd_strip_residual", "dH_gemm", "dW_gemm")
+
+
+def vp_ce_profile_enable(on: bool) -> None:
+    load_library().vp_ce_profile_enable(1 if on else 0)
+
+
+def vp_ce_profile_collect():
+    """Returns {kind: (total_ms, launches)} for the launches recorded since profiling was enabled."""
+    lib = load_library()
+    ms = (ctypes.c_double * 4)()
+    n = (ctypes.c_int64 * 4)()
+    _check(lib.vp_ce_profile_collect(ms, n))
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}

@@ -25,6 +25,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <mutex>
+#include <vector>
 
 #include "vp_ce.h"
 
@@ -590,6 +591,13 @@ __global__ void vpce_clear_status_kernel(int* status) { if (threadIdx.x < 8) sta
 // ------------------------------------------------------------------------------------ host side
 std::atomic<long long> g_launches{0};
 
+// Optional per-kernel timing: when enabled, every GEMM launch is bracketed by two events on the
+// launching stream; vp_ce_profile_collect sums the elapsed times per kernel kind.
+struct ProfEntry { int kind; cudaEvent_t a, b; };
+std::mutex g_prof_mu;
+bool g_prof_on = false;
+std::vector<ProfEntry> g_prof;
+
 struct WsLayout {
     size_t status, scalars, sm, sz, ylab, pm, pz, G, acc, total;
 };
@@ -669,7 +677,20 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const Ge
     const int tiles = p.m_tiles * p.n_tiles;
     if (tiles <= 0 || p.num_kb <= 0) return cudaSuccess;
     const int grid = tiles < num_sms() ? tiles : num_sms();
+    ProfEntry pe{EPI, nullptr, nullptr};
+    bool prof = false;
+    {
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        prof = g_prof_on;
+    }
+    if (prof && cudaEventCreate(&pe.a) == cudaSuccess && cudaEventCreate(&pe.b) == cudaSuccess) cudaEventRecord(pe.a, st);
+    else prof = false;
     kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmA, tmB, p);
+    if (prof) {
+        cudaEventRecord(pe.b, st);
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        g_prof.push_back(pe);
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError();
 }
@@ -889,6 +910,59 @@ vpce_status vp_ce_device_status(const void* workspace, int32_t* host_out, void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(host_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return VPCE_CUDA_ERROR;
+    return cudaStreamSynchronize(st) == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
+}
+
+void vp_ce_profile_enable(int on) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = on != 0;
+}
+
+vpce_status vp_ce_profile_collect(double* ms_out, int64_t* launches_out) {
+    if (!ms_out || !launches_out) return VPCE_INVALID_ARG;
+    std::vector<ProfEntry> entries;
+    {
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        entries.swap(g_prof);
+    }
+    for (int k = 0; k < 4; ++k) { ms_out[k] = 0.0; launches_out[k] = 0; }
+    vpce_status rc = VPCE_OK;
+    for (auto& e : entries) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(e.b) == cudaSuccess && cudaEventElapsedTime(&ms, e.a, e.b) == cudaSuccess) {
+            ms_out[e.kind] += ms;
+            launches_out[e.kind] += 1;
+        } else {
+            rc = VPCE_CUDA_ERROR;
+        }
+        cudaEventDestroy(e.a);
+        cudaEventDestroy(e.b);
+    }
+    return rc;
+}
+
+vpce_status vp_ce_fwd_bwd_host(const void* H_host, const int32_t* labels_host, const void* W, float* loss_host,
+                               void* dH_host, float* dW, int64_t T, int64_t d, int64_t V, int64_t block_v,
+                               int32_t ignore_index, int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW,
+                               void* H_dev, int32_t* labels_dev, float* loss_dev, float* lse_dev, void* dH_dev,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    if (!H_host || !labels_host || !loss_host || !dH_host || !H_dev || !labels_dev || !loss_dev || !lse_dev || !dH_dev)
+        return VPCE_INVALID_ARG;
+    if (T <= 0 || d <= 0) return VPCE_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t hbytes = static_cast<size_t>(T) * d * 2;
+    if (cudaMemcpyAsync(H_dev, H_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+    if (cudaMemcpyAsync(labels_dev, labels_host, static_cast<size_t>(T) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return VPCE_CUDA_ERROR;
+    vpce_status s = vp_ce_forward(H_dev, W, labels_dev, T, d, V, block_v, ignore_index, loss_dev, lse_dev, T_chunk,
+                                  chunk_index_base, workspace, workspace_bytes, stream);
+    if (s != VPCE_OK) return s;
+    s = vp_ce_backward(H_dev, W, labels_dev, lse_dev, nullptr, dH_dev, dW, T, d, V, block_v, ignore_index, T_chunk,
+                       chunk_index_base, accumulate_dW, workspace, workspace_bytes, stream);
+    if (s != VPCE_OK) return s;
+    if (cudaMemcpyAsync(loss_host, loss_dev, static_cast<size_t>(T) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return VPCE_CUDA_ERROR;
+    if (cudaMemcpyAsync(dH_host, dH_dev, hbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return VPCE_CUDA_ERROR;
     return cudaStreamSynchronize(st) == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
 }
 
