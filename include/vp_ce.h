@@ -47,6 +47,7 @@ typedef int vpce_status;
 #define VPCE_UNSUPPORTED         2  /* alignment or divisibility rule above not met           */
 #define VPCE_WORKSPACE_TOO_SMALL 3
 #define VPCE_CUDA_ERROR          4  /* a CUDA runtime/driver call or a launch failed          */
+#define VPCE_STATIC_SCRATCH_EXCEEDED 5  /* vp_ce_forward_static: sizes beyond its built-in scratch */
 
 /* Bits of the device status word (vp_ce_device_status). */
 #define VPCE_DEV_LABEL_OUT_OF_RANGE 1
@@ -129,6 +130,41 @@ vpce_status vp_ce_fwd_bwd_host(const void* H_host, const int32_t* labels_host, c
                                int32_t ignore_index, int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW,
                                void* H_dev, int32_t* labels_dev, float* loss_dev, float* lse_dev, void* dH_dev,
                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Forward for callers that can neither allocate device memory nor hand over a workspace.
+ * (The paper has no counterpart: its operator runs under a framework allocator.)
+ *
+ * Some callers of this library run where cudaMalloc is off limits: a plug-in that executes
+ * inside another runtime's memory plan (every device byte is owned by that runtime's arena and
+ * the plug-in may only touch the tensors it is handed), a step of a latency-critical serving
+ * loop where an allocation would synchronise the device, or code that runs after the process
+ * has deliberately filled the GPU.  For them this entry point computes exactly what
+ * vp_ce_forward computes, with the same kernels, but its scratch memory (per-token running
+ * state, per-tile partial states, status word) is a fixed array compiled into the library:
+ * VPCE_STATIC_SCRATCH_BYTES bytes of device memory that every GPU which loads the library
+ * holds until the process exits.
+ *
+ *   - Inputs and outputs are the caller's, as for vp_ce_forward.  device_status_out is an
+ *     optional DEVICE int32 that receives the status word (the bits VPCE_DEV_*) at the end of
+ *     the call; pass NULL to skip it.
+ *   - Limit: the forward part of the workspace layout for (T_chunk, block_v) must fit the
+ *     array, roughly 8 * T_chunk * (block_v / 256 + 2) bytes; T_chunk = 4096 with
+ *     block_v = 8192 fits.  Larger sizes return VPCE_STATIC_SCRATCH_EXCEEDED and launch
+ *     nothing; T, V and d are not limited by it.
+ *   - No cudaMalloc, cudaFree, event or stream creation or other allocating routine is called.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; the call
+ *     clears what must start at zero itself.  Two calls that overlap on the GPU (different
+ *     streams, or different host threads without ordering) race on it and give wrong results:
+ *     order them on one stream or with events.
+ */
+#define VPCE_STATIC_SCRATCH_BYTES (1280u * 1024u)
+vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* labels,
+                                 int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                                 float* loss, float* lse, int64_t T_chunk, int64_t chunk_index_base,
+                                 int32_t* device_status_out, void* stream);
 
 /*
  * Measurement aid (no counterpart in the paper).  While enabled, every tensor-core kernel

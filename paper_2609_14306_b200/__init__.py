@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     vp_ce_backward,
     vp_ce_device_status,
     vp_ce_forward,
+    vp_ce_forward_static,
     vp_ce_fwd_bwd_host,
     vp_ce_profile_collect,
     vp_ce_profile_enable,

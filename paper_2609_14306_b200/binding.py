@@ -54,6 +54,8 @@ def load_library() -> ctypes.CDLL:
     lib.vp_ce_fwd_bwd_host.restype = ctypes.c_int
     lib.vp_ce_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, i64, i64, ctypes.c_int,
                                        vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.vp_ce_forward_static.restype = ctypes.c_int
+    lib.vp_ce_forward_static.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, i64, i64, vp, vp]
     lib.vp_ce_profile_enable.restype = None
     lib.vp_ce_profile_enable.argtypes = [ctypes.c_int]
     lib.vp_ce_profile_collect.restype = ctypes.c_int
@@ -194,3 +196,19 @@ def vp_ce_profile_collect():
     n = (ctypes.c_int64 * 4)()
     _check(lib.vp_ce_profile_collect(ms, n))
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def vp_ce_forward_static(H, W, labels, block_v: int, ignore_index: int, loss, lse, T_chunk: int,
+                         chunk_index_base: int, device_status_out=None, stream=None) -> None:
+    """vp_ce_forward for callers that cannot allocate or pass a workspace: the scratch is a fixed
+    array inside the library (see include/vp_ce.h for its size limit and the sharing rules)."""
+    import torch
+    lib = load_library()
+    T, d, V = _shapes(H, W)
+    _check(lib.vp_ce_forward_static(
+        _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
+        T, d, V, int(block_v), int(ignore_index),
+        _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
+        int(T_chunk), int(chunk_index_base),
+        None if device_status_out is None else _ptr(device_status_out, torch.int32, "device_status_out", 1),
+        _stream_ptr(stream)))

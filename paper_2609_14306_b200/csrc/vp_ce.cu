@@ -748,6 +748,8 @@ const char* vp_ce_status_string(vpce_status s) {
         case VPCE_UNSUPPORTED: return "unsupported (alignment, d % 8, block_v % 256 or T_chunk % 128)";
         case VPCE_WORKSPACE_TOO_SMALL: return "workspace too small";
         case VPCE_CUDA_ERROR: return "CUDA error";
+        case VPCE_STATIC_SCRATCH_EXCEEDED:
+            return "T_chunk * block_v too large for the built-in scratch of vp_ce_forward_static";
         default: return "unknown status";
     }
 }
@@ -964,6 +966,116 @@ vpce_status vp_ce_fwd_bwd_host(const void* H_host, const int32_t* labels_host, c
         return VPCE_CUDA_ERROR;
     if (cudaMemcpyAsync(dH_host, dH_dev, hbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return VPCE_CUDA_ERROR;
     return cudaStreamSynchronize(st) == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
+}
+
+// ------------------------------------------------------------------------------------ forward without a caller workspace
+}  // extern "C"
+
+namespace {
+
+// Scratch of vp_ce_forward_static.  It is part of the loaded module: every GPU that loads this
+// library holds these bytes until the process exits.  In host code the NAME of a __device__
+// array is only a handle for the runtime, never an address a kernel may use; the device address
+// is looked up once per device with cudaGetSymbolAddress and that pointer is what kernels get.
+constexpr size_t STATIC_SCRATCH_BYTES = VPCE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[64] = {nullptr};
+
+// Device address of g_static_scratch on the current device (looked up on first use).
+vpce_status static_scratch_address(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VPCE_CUDA_ERROR;
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return VPCE_CUDA_ERROR;
+        g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return VPCE_OK;
+}
+
+__global__ void vpce_copy_status_kernel(const int* status, int* out) { if (threadIdx.x == 0) *out = *status; }
+
+}  // namespace
+
+extern "C" {
+
+vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
+                                 int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
+                                 int64_t chunk_index_base, int32_t* device_status_out, void* stream) {
+    if (!H || !W || !labels || !loss || !lse) return VPCE_INVALID_ARG;
+    if (T <= 0 || d <= 0 || V <= 0 || block_v <= 0 || T_chunk <= 0 || chunk_index_base < 0) return VPCE_INVALID_ARG;
+    if (!aligned16(H) || !aligned16(W)) return VPCE_UNSUPPORTED;
+    if (T >= (1ll << 31) || V >= (1ll << 31)) return VPCE_UNSUPPORTED;
+    WsLayout L;
+    if (!ws_layout(T_chunk, d, block_v, &L)) return VPCE_UNSUPPORTED;
+    // The forward touches the layout up to (not including) the residual strip G.
+    if (L.G > STATIC_SCRATCH_BYTES) return VPCE_STATIC_SCRATCH_EXCEEDED;
+    unsigned char* ws = nullptr;
+    vpce_status s = static_scratch_address(&ws);
+    if (s != VPCE_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* status = reinterpret_cast<int*>(ws + L.status);
+    float* sm = reinterpret_cast<float*>(ws + L.sm);
+    float* sz = reinterpret_cast<float*>(ws + L.sz);
+    float* ylab = reinterpret_cast<float*>(ws + L.ylab);
+    float* pm = reinterpret_cast<float*>(ws + L.pm);
+    float* pz = reinterpret_cast<float*>(ws + L.pz);
+
+    CUtensorMap tmH, tmW;
+    if (!make_map(&tmH, H, T, d, d, BK, BM) || !make_map(&tmW, W, V, d, d, BK, BN_VOCAB)) return VPCE_CUDA_ERROR;
+    using Cfg = StageCfg<BN_VOCAB>;
+    auto kern = vpce_gemm_kernel<BN_VOCAB, false, false, EPI_FOLD>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_TOTAL) != cudaSuccess)
+        return VPCE_CUDA_ERROR;
+
+    // The array keeps whatever the previous call left: the status word must start at zero; the
+    // running state is initialised by the first merge of every chunk and the partial slots are
+    // fully rewritten before they are read.
+    vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+
+    const int64_t P = (V + block_v - 1) / block_v;
+    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
+    const int num_kb = static_cast<int>((d + BK - 1) / BK);
+    for (int64_t c = 0; c < n_chunks; ++c) {
+        const int64_t tok0 = c * T_chunk;
+        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
+        const int64_t cg = chunk_index_base + c;
+        for (int64_t i = 0; i < P; ++i) {
+            const int64_t q = ((cg - i) % P + P) % P;
+            const int64_t v_lo = q * block_v;
+            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
+            GemmParams p{};
+            p.m_tiles = (rows + BM - 1) / BM;
+            p.n_tiles = (cols + BN_VOCAB - 1) / BN_VOCAB;
+            p.num_kb = num_kb;
+            p.a_mn0 = static_cast<int>(tok0); p.b_mn0 = static_cast<int>(v_lo);
+            p.rows_valid = rows; p.cols_valid = cols;
+            p.v_lo = static_cast<int>(v_lo);
+            p.labels = labels + tok0;
+            p.ignore_index = ignore_index; p.V = static_cast<int>(V);
+            p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
+            p.status = status;
+            const int tiles = p.m_tiles * p.n_tiles;
+            const int grid = tiles < num_sms() ? tiles : num_sms();
+            kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmH, tmW, p);
+            vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
+                                                                  rows, i == 0, i == P - 1, labels + tok0, ignore_index,
+                                                                  static_cast<int>(V), lse + tok0, loss + tok0, status);
+            g_launches.fetch_add(2, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return VPCE_CUDA_ERROR;
+        }
+    }
+    if (device_status_out) {
+        vpce_copy_status_kernel<<<1, 32, 0, st>>>(status, device_status_out);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return VPCE_CUDA_ERROR;
+    }
+    return VPCE_OK;
 }
 
 }  // extern "C"
