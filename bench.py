@@ -148,6 +148,28 @@ def run_reference(args, w):
     print(json.dumps(out), flush=True)
 
 
+# --------------------------------------------------------------------------- multi-rank helpers
+def rank_workload(w, rank: int):
+    """Rank r of a multi-GPU run draws its own batch stream (replicas on distinct data)."""
+    return w if rank == 0 else dataclasses.replace(w, seed=w.seed + 1000 * rank)
+
+
+def max_over_ranks(ms: float, device=None) -> float:
+    """MAX over ranks of a duration measured on each rank's device (identity on one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, tokens_per_rank: int, ms_max: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time."""
+    return world * tokens_per_rank / (ms_max / 1e3)
+
+
 # --------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -162,8 +184,8 @@ def main():
     ap.add_argument("--profile-in-timed-region", type=int, default=1)
     args = ap.parse_args()
 
-    from synth_inputs import IGNORE_INDEX, WORKLOADS, make_hidden, make_weights, stream_labels
-    w = WORKLOADS[args.workload]
+    from synth_inputs import IGNORE_INDEX, PROFILE_WORKLOADS, WORKLOADS, make_hidden, make_weights, stream_labels
+    w = WORKLOADS.get(args.workload) or PROFILE_WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -196,8 +218,7 @@ def main():
     H_host0 = make_hidden(w, 0) if rank == 0 else None
     Hs, labs = [], []
     for call in range(w.n_calls):
-        hb = H_host0 if (call == 0 and rank == 0) else make_hidden(
-            w if rank == 0 else dataclasses.replace(w, seed=w.seed + 1000 * rank), call)
+        hb = H_host0 if (call == 0 and rank == 0) else make_hidden(rank_workload(w, rank), call)
         Hs.append(bf16_dev(hb))
         labs.append(torch.from_numpy(labels_all[call * w.T:(call + 1) * w.T].copy()).to(dev))
     n_valid_total = int((labels_all != IGNORE_INDEX).sum())
@@ -255,11 +276,7 @@ def main():
     prof = vp.vp_ce_profile_collect() if prof_on else None
     launches = vp.vp_ce_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
     peak_extra = torch.cuda.max_memory_allocated(dev) - resident
     mean_loss = float(mean.item())
@@ -292,14 +309,8 @@ def main():
         for _ in range(args.steps):
             e2e_step()
         e1.record(); barrier()
-        ms_e2e = e0.elapsed_time(e1)
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        ms_e2e /= args.steps
-        e2e = {"value": world * w.T_stream / (ms_e2e / 1e3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+        e2e = {"value": whole_job_tokens_per_s(world, w.T_stream, ms_e2e), "unit": "tokens/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": w.T * w.d * 2 + w.T * 4, "d2h_bytes_per_step": w.T * 4 + w.T * w.d * 2,
                "api": "vp_ce_fwd_bwd_host (pinned host H, labels in; loss, dH out; W and dW resident)",
                "mean_loss_host": float(loss_h[lh != IGNORE_INDEX].double().mean())}
@@ -312,7 +323,7 @@ def main():
 
     peaks, peak_src = load_peaks()
     tokens = w.T_stream
-    value = world * tokens / (ms_step / 1e3)
+    value = whole_job_tokens_per_s(world, tokens, ms_step)
     tflops = w.flops / (ms_step / 1e3) / 1e12
     out = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,

@@ -10,9 +10,10 @@ random hidden states with H=7168 and V=200000 and describes no targets).
 
 Recipe
 ------
-* one ``numpy.random.Generator(PCG64)`` per array, seeded by
-  ``SeedSequence([seed, stream_id, call_index])`` (stream ids below), so arrays are
-  independent and any call of a streamed workload can be regenerated alone;
+* one ``numpy.random.Generator(PCG64)`` per array (labels, masks) or per slab of 4096 rows
+  (H, W), seeded by ``SeedSequence([seed, stream_id, call_index(, slab)])`` (stream ids below),
+  so arrays are independent, slabs can be drawn by several threads with the same result, and
+  any call of a streamed workload can be regenerated alone;
 * H ~ N(0, 1), W ~ N(0, w_std^2): float32 normals scaled in float32, then rounded to bf16;
 * labels: uniform over [0, V) or truncated Zipf(s) over ranks 1..V with id = rank-1,
   sampled by inverse CDF (float64 ``searchsorted``);
@@ -23,6 +24,8 @@ from __future__ import annotations
 
 import dataclasses
 import hashlib
+import os
+from concurrent.futures import ThreadPoolExecutor
 from typing import Dict, Optional
 
 import numpy as np
@@ -98,6 +101,19 @@ WORKLOADS: Dict[str, Workload] = {
 }
 
 
+# Reduced cases of the moe120b / moe667b shapes for profiler captures: operands larger than the
+# 126 MB L2 but well under a gigabyte on the device, a few launches per kernel kind.
+PROFILE_WORKLOADS: Dict[str, Workload] = {
+    w.name: w
+    for w in [
+        Workload("prof120b", T=4096, d=2880, V=32768, block_v=8192, T_chunk=4096,
+                 w_std=0.02, labels="zipf", zipf_s=1.1, ignore_frac=0.05, seed=12),
+        Workload("prof667b", T=4096, d=7168, V=16384, block_v=8192, T_chunk=4096,
+                 w_std=0.006, labels="zipf", zipf_s=1.1, ignore_frac=0.02, seed=13),
+    ]
+}
+
+
 # --------------------------------------------------------------------------- bf16 helpers
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round float32 to bfloat16 (nearest, ties to even); returns the uint16 bit patterns."""
@@ -113,8 +129,19 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
 
 
 def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
-    """Widen bfloat16 bit patterns to float64 exactly."""
-    return bf16_bits_to_f32(bits).astype(np.float64)
+    """Widen bfloat16 bit patterns to float64 exactly (row slabs in a thread pool when large)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    if bits.ndim != 2 or bits.size < (1 << 24):
+        return bf16_bits_to_f32(bits).astype(np.float64)
+    out = np.empty(bits.shape, dtype=np.float64)
+    step = max(1, (1 << 22) // bits.shape[1])
+
+    def conv(r0: int) -> None:
+        out[r0:r0 + step] = bf16_bits_to_f32(bits[r0:r0 + step])
+
+    with ThreadPoolExecutor(max(1, min(16, os.cpu_count() or 1))) as ex:
+        list(ex.map(conv, range(0, bits.shape[0], step)))
+    return out
 
 
 # --------------------------------------------------------------------------- generators
@@ -122,22 +149,38 @@ def _rng(seed: int, stream: int, call_index: int) -> np.random.Generator:
     return np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, stream, call_index])))
 
 
-def gaussian_bf16(shape, std: float, seed: int, stream: int, call_index: int = 0,
-                  slab_rows: int = 8192) -> np.ndarray:
+SLAB_ROWS = 4096       # part of the recipe: each slab of rows has its own generator
+
+
+def _threads() -> int:
+    return max(1, min(16, os.cpu_count() or 1))
+
+
+def gaussian_bf16(shape, std: float, seed: int, stream: int, call_index: int = 0) -> np.ndarray:
     """N(0, std^2) draws rounded to bf16, returned as uint16 bit patterns of ``shape``.
 
-    Rows are drawn slab by slab from one generator so peak host memory stays small.
+    Slab k (rows [k*SLAB_ROWS, (k+1)*SLAB_ROWS)) is drawn from its own generator
+    SeedSequence([seed, stream, call_index, k]); slabs are filled by a thread pool, and the
+    result does not depend on the number of threads.
     """
     rows, cols = int(shape[0]), int(shape[1])
     out = np.empty((rows, cols), dtype=np.uint16)
-    rng = _rng(seed, stream, call_index)
     s = np.float32(std)
-    for r0 in range(0, rows, slab_rows):
-        r1 = min(rows, r0 + slab_rows)
+
+    def fill(k: int) -> None:
+        r0, r1 = k * SLAB_ROWS, min(rows, (k + 1) * SLAB_ROWS)
+        rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, stream, call_index, k])))
         x = rng.standard_normal((r1 - r0, cols), dtype=np.float32)
         if std != 1.0:
             x *= s
         out[r0:r1] = f32_to_bf16_bits(x)
+
+    n_slabs = -(-rows // SLAB_ROWS)
+    if n_slabs == 1:
+        fill(0)
+    else:
+        with ThreadPoolExecutor(_threads()) as ex:
+            list(ex.map(fill, range(n_slabs)))
     return out
 
 
