@@ -179,13 +179,22 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="moe120b")
     ap.add_argument("--t-chunk", type=int, default=0)
+    ap.add_argument("--shape", default="", help="custom workload T,d,V,block_v (Gaussian inputs, Zipf labels); "
+                                                "for kernel experiments, not a benchmark config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-in-timed-region", type=int, default=1)
     args = ap.parse_args()
 
     from synth_inputs import IGNORE_INDEX, PROFILE_WORKLOADS, WORKLOADS, make_hidden, make_weights, stream_labels
-    w = WORKLOADS.get(args.workload) or PROFILE_WORKLOADS[args.workload]
+    if args.shape:
+        from synth_inputs import custom_workload
+        T_, d_, V_, bv_ = (int(x) for x in args.shape.split(","))
+        w = custom_workload("custom", T=T_, d=d_, V=V_, block_v=bv_, T_chunk=args.t_chunk or T_, w_std=0.02,
+                            labels="zipf", ignore_frac=0.05, seed=99)
+        args.workload = "custom"
+    else:
+        w = WORKLOADS.get(args.workload) or PROFILE_WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
         return
