@@ -24,6 +24,7 @@
 #include <atomic>
 #include <cstdint>
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
 #include <vector>
 
@@ -39,12 +40,16 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_WARP0 = 2;
 constexpr int SMEM_BUDGET = 200 * 1024;    // operand stages
 constexpr int SMEM_EXTRA = 2048;           // barriers + alignment slack
+constexpr int G_STAGING_BYTES = 4 * 2 * 4096;   // RESID: per epilogue warp two 32-row x 64-column bf16 boxes
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
 
 enum Epilogue { EPI_FOLD = 0, EPI_RESID = 1, EPI_DH = 2, EPI_DW = 3 };
 
 struct GemmParams {
     int m_tiles, n_tiles, num_kb;
+    int a_3d, b_3d;                        // MN-major operand fetched as one 3-D box (64 x 64 x chunks) per k-block
+    int hint_a, hint_b, hint_c;            // L2 eviction hints for A loads, B loads, C stores: 0 normal, 1 first, 2 last
+    int group_n;                           // n-tiles per raster group (tiles run m-major inside a group)
     int a_mn0, a_k0, b_mn0, b_k0;          // TMA coordinate bases (elements)
     int rows_valid;                        // valid accumulator rows overall (M bound)
     int cols_valid;                        // valid accumulator columns overall (N bound)
@@ -126,6 +131,46 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint64_t make_policy(int kind) {
+    uint64_t pol;
+    if (kind == 1) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    else if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, uint32_t src, int c0, int c1, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -196,11 +241,28 @@ template <int BN> struct StageCfg {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
     static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
+    // the residual epilogue stages its bf16 tile in shared memory for TMA stores
+    static constexpr int SMEM_TOTAL_STAGED = SMEM_TOTAL + G_STAGING_BYTES;
 };
+template <int BN, int EPI> constexpr int smem_total() {
+    return EPI == 1 ? StageCfg<BN>::SMEM_TOTAL_STAGED : StageCfg<BN>::SMEM_TOTAL;
+}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// Tile order: the n-tiles are cut into groups of group_n; inside a group the index runs n-fastest
+// over all m-tiles, so the group's B operand (a slice of the shard) stays in L2 while A streams.
+__device__ __forceinline__ void decode_tile(const GemmParams& p, int tile, int& mt, int& nt) {
+    const int per_group = p.group_n * p.m_tiles;
+    const int g = tile / per_group;
+    const int r = tile - g * per_group;
+    const int n0 = g * p.group_n;
+    const int gw = min(p.group_n, p.n_tiles - n0);
+    mt = r / gw;
+    nt = n0 + (r - mt * gw);
 }
 
 // ------------------------------------------------------------------------------------ epilogues
@@ -251,7 +313,11 @@ __device__ __forceinline__ void epilogue_fold(const GemmParams& p, int mt, int n
     }
 }
 
-__device__ __forceinline__ void epilogue_resid(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+// The bf16 residual tile leaves through shared memory: each epilogue warp owns 32 rows; per 64
+// columns it fills a 32 x 128-byte box (128-byte swizzle: 16-byte chunk j of row r sits at chunk
+// j ^ (r & 7)) and one lane issues a TMA store, so global writes are whole 128-byte lines.
+__device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtensorMap* tmG, uint32_t stage_smem,
+                                               int mt, int nt, int row, int lane, uint32_t tmem_row) {
     const int grow = mt * BM + row;
     const bool row_ok = grow < p.rows_valid;
     int label = row_ok ? p.labels[grow] : p.ignore_index;
@@ -260,30 +326,44 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, int mt, int 
     if (valid) dl = p.dloss ? p.dloss[grow] : *p.inv_n_valid;
     if (row_ok) lseL = p.lse[grow] * LOG2E;
     const int lrel = valid ? label - (p.v_lo + nt * BN_VOCAB) : -1;
-    __nv_bfloat16* grow_ptr = p.G + static_cast<size_t>(grow) * p.g_ld + nt * BN_VOCAB;
+    const uint64_t pol_c = make_policy(p.hint_c);
 #pragma unroll 1
-    for (int c = 0; c < BN_VOCAB / 32; ++c) {
-        float v[32];
+    for (int h = 0; h < BN_VOCAB / 64; ++h) {
+        const uint32_t buf = stage_smem + (h & 1) * 4096;
+        if (lane == 0) bulk_wait_read_1();                              // the store that last read this buffer is done
         __syncwarp();
-        tmem_ld32(tmem_row + c * 32, v);
-        tmem_ld_wait();
-        const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);
-        const int jj = lrel - c * 32;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            float g = dl * ex2f(fmaf(v[j], LOG2E, -lseL));
-            if (j == jj) g -= dl;
-            v[j] = (j < nvalid) ? g : 0.f;
+        for (int c2 = 0; c2 < 2; ++c2) {
+            const int c = 2 * h + c2;
+            float v[32];
+            __syncwarp();
+            tmem_ld32(tmem_row + c * 32, v);
+            tmem_ld_wait();
+            const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);
+            const int jj = lrel - c * 32;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                float g = dl * ex2f(fmaf(v[j], LOG2E, -lseL));
+                if (j == jj) g -= dl;
+                v[j] = (j < nvalid) ? g : 0.f;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint4 o;
+                o.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
+                o.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
+                o.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
+                o.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
+                const int chunk = c2 * 4 + q;                           // 16-byte chunk within the 128-byte row
+                st_shared_v4(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4), o);   // rows >= rows_valid get zeros
+            }
         }
-        uint4* dst = reinterpret_cast<uint4*>(grow_ptr + c * 32);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint4 o;
-            o.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
-            o.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
-            o.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
-            o.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
-            dst[q] = o;                                                // rows >= rows_valid get zeros
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+            if (p.hint_c) tma_store_2d_hint(tmG, buf, nt * BN_VOCAB + h * 64, mt * BM + (row - lane), pol_c);
+            else tma_store_2d(tmG, buf, nt * BN_VOCAB + h * 64, mt * BM + (row - lane));
+            bulk_commit();
         }
     }
 }
@@ -356,7 +436,8 @@ __device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt,
 // ------------------------------------------------------------------------------------ the GEMM kernel
 template <int BN, bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
     using Cfg = StageCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr uint32_t TMEM_COLS = (BN > 128) ? 512u : (BN > 64 ? 256u : 128u);
@@ -375,6 +456,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const uint32_t g_staging = base + STAGES * Cfg::STAGE_BYTES + 1024;   // RESID only (1024-byte aligned)
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -404,27 +486,51 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             long issued = 0;
+            const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
+            const bool use_a = p.hint_a != 0, use_b = p.hint_b != 0;
+            auto load_a = [&](uint32_t dst, uint32_t bar, int c0, int c1) {
+                if (use_a) tma_load_2d_hint(dst, &tmA, bar, c0, c1, pol_a); else tma_load_2d(dst, &tmA, bar, c0, c1);
+            };
+            auto load_b = [&](uint32_t dst, uint32_t bar, int c0, int c1) {
+                if (use_b) tma_load_2d_hint(dst, &tmB, bar, c0, c1, pol_b); else tma_load_2d(dst, &tmB, bar, c0, c1);
+            };
+            // The loads of one k-block of one tile into a stage.
+            auto issue = [&](int mt, int nt, int kb, uint32_t sa, uint32_t sb, uint32_t bar) {
+                if (A_MN && p.a_3d) {
+                    const int c1 = p.a_k0 + kb * BK, c2 = (p.a_mn0 + mt * BM) >> 6;
+                    if (use_a) tma_load_3d_hint(sa, &tmA, bar, 0, c1, c2, pol_a); else tma_load_3d(sa, &tmA, bar, 0, c1, c2);
+                } else if (A_MN) {
+#pragma unroll
+                    for (int j = 0; j < BM / 64; ++j) {
+                        const int c0 = p.a_mn0 + mt * BM + 64 * j, c1 = p.a_k0 + kb * BK;
+                        load_a(sa + j * (BK * 128), bar, c0, c1);
+                    }
+                } else {
+                    const int c0 = p.a_k0 + kb * BK, c1 = p.a_mn0 + mt * BM;
+                    load_a(sa, bar, c0, c1);
+                }
+                if (B_MN && p.b_3d) {
+                    const int c1 = p.b_k0 + kb * BK, c2 = (p.b_mn0 + nt * BN) >> 6;
+                    if (use_b) tma_load_3d_hint(sb, &tmB, bar, 0, c1, c2, pol_b); else tma_load_3d(sb, &tmB, bar, 0, c1, c2);
+                } else if (B_MN) {
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j) {
+                        const int c0 = p.b_mn0 + nt * BN + 64 * j, c1 = p.b_k0 + kb * BK;
+                        load_b(sb + j * (BK * 128), bar, c0, c1);
+                    }
+                } else {
+                    const int c0 = p.b_k0 + kb * BK, c1 = p.b_mn0 + nt * BN;
+                    load_b(sb, bar, c0, c1);
+                }
+            };
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+                int mt, nt;
+                decode_tile(p, tile, mt, nt);
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-                    const uint32_t sb = sa + Cfg::A_BYTES;
-                    if (A_MN) {
-#pragma unroll
-                        for (int j = 0; j < BM / 64; ++j)
-                            tma_load_2d(sa + j * (BK * 128), &tmA, full_bar(stage), p.a_mn0 + mt * BM + 64 * j, p.a_k0 + kb * BK);
-                    } else {
-                        tma_load_2d(sa, &tmA, full_bar(stage), p.a_k0 + kb * BK, p.a_mn0 + mt * BM);
-                    }
-                    if (B_MN) {
-#pragma unroll
-                        for (int j = 0; j < BN / 64; ++j)
-                            tma_load_2d(sb + j * (BK * 128), &tmB, full_bar(stage), p.b_mn0 + nt * BN + 64 * j, p.b_k0 + kb * BK);
-                    } else {
-                        tma_load_2d(sb, &tmB, full_bar(stage), p.b_k0 + kb * BK, p.b_mn0 + nt * BN);
-                    }
+                    issue(mt, nt, kb, sa, sa + Cfg::A_BYTES, full_bar(stage));
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -482,20 +588,22 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int row = quad * 32 + lane;
         int it = 0; bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-            const int mt = tile / p.n_tiles, nt = tile % p.n_tiles;
+            int mt, nt;
+                decode_tile(p, tile, mt, nt);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
             if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
-            else if (EPI == EPI_RESID) epilogue_resid(p, mt, nt, row, tmem_row);
+            else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
             else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row);
             else epilogue_dw<BN>(p, mt, nt, row, tmem_row);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(ab));
         }
+        if (EPI == EPI_RESID && lane == 0) bulk_wait_all();             // staged stores have landed
     }
 
     tc_fence_before();
@@ -650,6 +758,22 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
     return r == CUDA_SUCCESS;
 }
 
+// MN-major operand of a row-major [k_rows, mn_cols] matrix (mn_cols % 64 == 0) as a 3-D tensor
+// {64 contiguous elements, k_rows, mn_cols / 64}: one box {64, 64, chunks} per k-block lands in
+// shared memory as `chunks` consecutive 64 x 128-byte blocks, the layout the MMA descriptor expects.
+bool make_map_mn3d(CUtensorMap* map, const void* ptr, uint64_t k_rows, uint64_t mn_cols, uint64_t ld_elems, uint32_t chunks) {
+    auto enc = get_encode();
+    if (!enc || mn_cols % 64) return false;
+    cuuint64_t dims[3] = {64, k_rows, mn_cols / 64};
+    cuuint64_t strides[2] = {ld_elems * 2, 128};
+    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(BK), chunks};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 int num_sms() {
     static int cached[64] = {0};
     int dev = 0;
@@ -663,14 +787,15 @@ int num_sms() {
 }
 
 template <int BN, bool A_MN, bool B_MN, int EPI>
-cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
-    using Cfg = StageCfg<BN>;
+cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const GemmParams& p,
+                        cudaStream_t st) {
+    constexpr int SMEM = smem_total<BN, EPI>();
     auto kern = vpce_gemm_kernel<BN, A_MN, B_MN, EPI>;
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_TOTAL);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
@@ -685,7 +810,7 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const Ge
     }
     if (prof && cudaEventCreate(&pe.a) == cudaSuccess && cudaEventCreate(&pe.b) == cudaSuccess) cudaEventRecord(pe.a, st);
     else prof = false;
-    kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmA, tmB, p);
+    kern<<<grid, NUM_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
     if (prof) {
         cudaEventRecord(pe.b, st);
         std::lock_guard<std::mutex> lk(g_prof_mu);
@@ -710,11 +835,31 @@ int pick_bn(int64_t d) {
 template <bool A_MN, bool B_MN, int EPI>
 cudaError_t launch_grad(int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
     switch (bn) {
-        case 256: return launch_gemm<256, A_MN, B_MN, EPI>(tmA, tmB, p, st);
-        case 192: return launch_gemm<192, A_MN, B_MN, EPI>(tmA, tmB, p, st);
-        case 128: return launch_gemm<128, A_MN, B_MN, EPI>(tmA, tmB, p, st);
-        default:  return launch_gemm<64, A_MN, B_MN, EPI>(tmA, tmB, p, st);
+        case 256: return launch_gemm<256, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
+        case 192: return launch_gemm<192, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
+        case 128: return launch_gemm<128, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
+        default:  return launch_gemm<64, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
     }
+}
+
+// n-tiles per raster group: the B operand slice a group touches should stay L2-resident
+// (<= ~48 MB), and groups are balanced.
+int pick_group_n(int n_tiles, double b_total_bytes) {
+    const double budget = 48.0 * 1024 * 1024;
+    int groups = static_cast<int>((b_total_bytes + budget - 1) / budget);
+    if (groups < 1) groups = 1;
+    if (groups > n_tiles) groups = n_tiles;
+    return (n_tiles + groups - 1) / groups;
+}
+
+// L2 eviction hints: the shard-side operand B is reused by every m-tile (keep it), the residual
+// strip G is streamed out by RESID and streamed in by the two gradient GEMMs (let it go first).
+void apply_tuning(GemmParams& p, int epi) {
+    p.hint_a = 0;
+    p.hint_b = 2;
+    p.hint_c = (epi == EPI_RESID) ? 1 : 0;
+    const char* e = getenv("VPCE_HINTS");
+    if (e) { int hv = atoi(e); p.hint_a = hv / 100; p.hint_b = (hv / 10) % 10; p.hint_c = hv % 10; }
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -793,6 +938,7 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
             p.m_tiles = (rows + BM - 1) / BM;
             p.n_tiles = (cols + BN_VOCAB - 1) / BN_VOCAB;
             p.num_kb = num_kb;
+            p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * d);
             p.a_mn0 = static_cast<int>(tok0); p.a_k0 = 0;
             p.b_mn0 = static_cast<int>(v_lo); p.b_k0 = 0;
             p.rows_valid = rows; p.cols_valid = cols;
@@ -801,7 +947,8 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
             p.ignore_index = ignore_index; p.V = static_cast<int>(V);
             p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
             p.status = status;
-            if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            apply_tuning(p, EPI_FOLD);
+            if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, tmH, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
                                                                   rows, i == 0, i == P - 1, labels + tok0, ignore_index,
                                                                   static_cast<int>(V), lse + tok0, loss + tok0, status);
@@ -828,8 +975,9 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
     __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.G);
     float* acc = reinterpret_cast<float*>(ws + L.acc);
 
-    CUtensorMap tmH_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmH_mn;
-    if (!make_map(&tmH_k, H, T, d, d, BK, BM) || !make_map(&tmW_k, W, V, d, d, BK, BN_VOCAB) ||
+    CUtensorMap tmH_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmH_mn, tmG_st;
+    if (!make_map(&tmG_st, G, T_chunk, block_v, block_v, 64, 32) ||
+        !make_map(&tmH_k, H, T, d, d, BK, BM) || !make_map(&tmW_k, W, V, d, d, BK, BN_VOCAB) ||
         !make_map(&tmG_k, G, T_chunk, block_v, block_v, BK, BM) || !make_map(&tmW_mn, W, V, d, d, 64, BK) ||
         !make_map(&tmG_mn, G, T_chunk, block_v, block_v, 64, BK) || !make_map(&tmH_mn, H, T, d, d, 64, BK))
         return VPCE_CUDA_ERROR;
@@ -842,6 +990,13 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
     }
 
     const int bn = pick_bn(d);
+    // one-instruction fetch of MN-major operands when the contiguous extent is a multiple of 64
+    const bool mn3d = (d % 64 == 0);
+    if (mn3d) {
+        if (!make_map_mn3d(&tmW_mn, W, V, d, d, bn / 64) || !make_map_mn3d(&tmH_mn, H, T, d, d, bn / 64) ||
+            !make_map_mn3d(&tmG_mn, G, T_chunk, block_v, block_v, BM / 64))
+            return VPCE_CUDA_ERROR;
+    }
     const int64_t P = (V + block_v - 1) / block_v;
     const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
     for (int64_t c = 0; c < n_chunks; ++c) {
@@ -858,6 +1013,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             p.m_tiles = (rows + BM - 1) / BM;
             p.n_tiles = strip_tiles_n;
             p.num_kb = static_cast<int>((d + BK - 1) / BK);
+            p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * d);
             p.a_mn0 = static_cast<int>(tok0); p.b_mn0 = static_cast<int>(v_lo);
             p.rows_valid = rows; p.cols_valid = cols;
             p.v_lo = static_cast<int>(v_lo);
@@ -865,7 +1021,8 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             p.inv_n_valid = inv_n; p.ignore_index = ignore_index; p.V = static_cast<int>(V);
             p.G = G; p.g_ld = static_cast<int>(block_v);
             p.status = status;
-            if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            apply_tuning(p, EPI_RESID);
+            if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, tmG_st, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             const int k_cols = strip_tiles_n * BN_VOCAB;               // columns of G written by step (1)
             const int m_rows = p.m_tiles * BM;                         // rows of G written by step (1)
             // (2) dH_c += G W_q : M = tokens, N = d, K = shard vocabulary
@@ -873,6 +1030,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             ph.m_tiles = p.m_tiles;
             ph.n_tiles = static_cast<int>((d + bn - 1) / bn);
             ph.num_kb = k_cols / BK;
+            ph.group_n = pick_group_n(ph.n_tiles, 2.0 * k_cols * d);
             ph.a_mn0 = 0; ph.a_k0 = 0;
             ph.b_mn0 = 0; ph.b_k0 = static_cast<int>(v_lo);
             ph.rows_valid = rows; ph.cols_valid = static_cast<int>(d);
@@ -880,18 +1038,23 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             ph.dH = static_cast<__nv_bfloat16*>(dH) + tok0 * d; ph.out_ld = static_cast<int>(d);
             ph.first = (i == 0); ph.last = (i == P - 1);
             ph.status = status;
+            ph.b_3d = mn3d;
+            apply_tuning(ph, EPI_DH);
             if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             // (3) dW_q += G^T H_c : M = shard vocabulary, N = d, K = chunk tokens
             GemmParams pw{};
             pw.m_tiles = (cols + BM - 1) / BM;
             pw.n_tiles = ph.n_tiles;
             pw.num_kb = m_rows / BK;
+            pw.group_n = pick_group_n(pw.n_tiles, 2.0 * m_rows * d);
             pw.a_mn0 = 0; pw.a_k0 = 0;
             pw.b_mn0 = 0; pw.b_k0 = static_cast<int>(tok0);
             pw.rows_valid = cols; pw.cols_valid = static_cast<int>(d);
             pw.dW = dW + v_lo * d; pw.out_ld = static_cast<int>(d);
             pw.accumulate = (accumulate_dW != 0) || (c > 0);
             pw.status = status;
+            pw.a_3d = mn3d; pw.b_3d = mn3d;
+            apply_tuning(pw, EPI_DW);
             if (launch_grad<true, true, EPI_DW>(bn, tmG_mn, tmH_mn, pw, st) != cudaSuccess) return VPCE_CUDA_ERROR;
         }
     }
@@ -1053,6 +1216,7 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
             p.m_tiles = (rows + BM - 1) / BM;
             p.n_tiles = (cols + BN_VOCAB - 1) / BN_VOCAB;
             p.num_kb = num_kb;
+            p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * d);
             p.a_mn0 = static_cast<int>(tok0); p.b_mn0 = static_cast<int>(v_lo);
             p.rows_valid = rows; p.cols_valid = cols;
             p.v_lo = static_cast<int>(v_lo);
@@ -1060,9 +1224,10 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
             p.ignore_index = ignore_index; p.V = static_cast<int>(V);
             p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
             p.status = status;
+            apply_tuning(p, EPI_FOLD);
             const int tiles = p.m_tiles * p.n_tiles;
             const int grid = tiles < num_sms() ? tiles : num_sms();
-            kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmH, tmW, p);
+            kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmH, tmW, tmH, p);
             vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
                                                                   rows, i == 0, i == P - 1, labels + tok0, ignore_index,
                                                                   static_cast<int>(V), lse + tok0, loss + tok0, status);
