@@ -37,7 +37,6 @@ constexpr int BK = 64;           // K elements per pipeline stage (one 128-byte 
 constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
 constexpr int BN_VOCAB = 256;    // vocabulary columns per strip tile
 constexpr int NUM_THREADS = 192;
-constexpr int EPI_WARP0 = 2;
 constexpr int SMEM_BUDGET = 200 * 1024;    // operand stages
 constexpr int SMEM_EXTRA = 2048;           // barriers + alignment slack
 constexpr int G_STAGING_BYTES = 4 * 2 * 4096;   // RESID: per epilogue warp two 32-row x 64-column bf16 boxes
@@ -77,6 +76,7 @@ struct GemmParams {
     int accumulate;
     int out_ld;
     int* status;
+    int* tile_counter;                     // zero before the launch; tiles are taken with atomicAdd
 };
 
 // ------------------------------------------------------------------------------------ PTX wrappers
@@ -369,11 +369,11 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtens
 }
 
 template <int BN>
-__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row, int n_this) {
     const int grow = mt * BM + row;
     const bool row_ok = grow < p.rows_valid;
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
+    for (int c = 0; c < (n_this + 31) / 32; ++c) {
         float v[32];
         __syncwarp();
         tmem_ld32(tmem_row + c * 32, v);
@@ -407,11 +407,11 @@ __device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt,
 }
 
 template <int BN>
-__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
+__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row, int n_this) {
     const int grow = mt * BM + row;                                    // vocabulary row within the shard
     const bool row_ok = grow < p.rows_valid;
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
+    for (int c = 0; c < (n_this + 31) / 32; ++c) {
         float v[32];
         __syncwarp();
         tmem_ld32(tmem_row + c * 32, v);
@@ -434,6 +434,13 @@ __device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt,
 }
 
 // ------------------------------------------------------------------------------------ the GEMM kernel
+// Tiles are handed out dynamically: the producer lane takes the next tile index from a global
+// counter (atomicAdd) and publishes it to the MMA lane and the epilogue warps through a small
+// shared-memory ring guarded by mbarriers, so a CTA that finishes early simply takes more tiles.
+// The last n-tile of a row may be narrower than BN (its MMA uses N = valid columns rounded up
+// to 16), so an output width that is not a multiple of BN costs no padded tensor-core work.
+constexpr int SCHED_DEPTH = 4;
+
 template <int BN, bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -442,7 +449,6 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int STAGES = Cfg::STAGES;
     constexpr uint32_t TMEM_COLS = (BN > 128) ? 512u : (BN > 64 ? 256u : 128u);
     constexpr uint32_t ACC_STRIDE = TMEM_COLS / 2;
-    constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -454,8 +460,12 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
     const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 5));
+    auto sfull_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + s); };
+    auto sempty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + SCHED_DEPTH + s); };
+    constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * SCHED_DEPTH;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* sched_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [SCHED_DEPTH] tile ids
     const uint32_t g_staging = base + STAGES * Cfg::STAGE_BYTES + 1024;   // RESID only (1024-byte aligned)
 
     const int warp = threadIdx.x >> 5;
@@ -467,6 +477,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
         mbar_init(drain_bar, 1);
+        for (int s = 0; s < SCHED_DEPTH; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 5); }
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tensormap(&tmA);
@@ -481,10 +492,17 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Valid accumulator columns of n-tile nt, rounded up to the MMA's granularity of 16.
+    auto tile_n = [&](int nt) {
+        const int left = p.cols_valid - nt * BN;
+        return left >= BN ? BN : ((left + 15) & ~15);
+    };
+
     if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
+        // ---------------------------------------------------------------- scheduler + TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
+            int ss = 0; uint32_t sphase = 0;
             long issued = 0;
             const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
             const bool use_a = p.hint_a != 0, use_b = p.hint_b != 0;
@@ -501,29 +519,30 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (use_a) tma_load_3d_hint(sa, &tmA, bar, 0, c1, c2, pol_a); else tma_load_3d(sa, &tmA, bar, 0, c1, c2);
                 } else if (A_MN) {
 #pragma unroll
-                    for (int j = 0; j < BM / 64; ++j) {
-                        const int c0 = p.a_mn0 + mt * BM + 64 * j, c1 = p.a_k0 + kb * BK;
-                        load_a(sa + j * (BK * 128), bar, c0, c1);
-                    }
+                    for (int j = 0; j < BM / 64; ++j)
+                        load_a(sa + j * (BK * 128), bar, p.a_mn0 + mt * BM + 64 * j, p.a_k0 + kb * BK);
                 } else {
-                    const int c0 = p.a_k0 + kb * BK, c1 = p.a_mn0 + mt * BM;
-                    load_a(sa, bar, c0, c1);
+                    load_a(sa, bar, p.a_k0 + kb * BK, p.a_mn0 + mt * BM);
                 }
                 if (B_MN && p.b_3d) {
                     const int c1 = p.b_k0 + kb * BK, c2 = (p.b_mn0 + nt * BN) >> 6;
                     if (use_b) tma_load_3d_hint(sb, &tmB, bar, 0, c1, c2, pol_b); else tma_load_3d(sb, &tmB, bar, 0, c1, c2);
                 } else if (B_MN) {
 #pragma unroll
-                    for (int j = 0; j < BN / 64; ++j) {
-                        const int c0 = p.b_mn0 + nt * BN + 64 * j, c1 = p.b_k0 + kb * BK;
-                        load_b(sb + j * (BK * 128), bar, c0, c1);
-                    }
+                    for (int j = 0; j < BN / 64; ++j)
+                        load_b(sb + j * (BK * 128), bar, p.b_mn0 + nt * BN + 64 * j, p.b_k0 + kb * BK);
                 } else {
-                    const int c0 = p.b_k0 + kb * BK, c1 = p.b_mn0 + nt * BN;
-                    load_b(sb, bar, c0, c1);
+                    load_b(sb, bar, p.b_k0 + kb * BK, p.b_mn0 + nt * BN);
                 }
             };
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            while (ok) {
+                if (!mbar_wait(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; break; }
+                int tile = atomicAdd(p.tile_counter, 1);
+                if (tile >= total_tiles) tile = -1;
+                sched_slot[ss] = tile;
+                mbar_arrive(sfull_bar(ss));                              // release: the slot is visible to waiters
+                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+                if (tile < 0) break;
                 int mt, nt;
                 decode_tile(p, tile, mt, nt);
                 for (int kb = 0; kb < p.num_kb; ++kb) {
@@ -550,8 +569,16 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            int it = 0;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+            int ss = 0; uint32_t sphase = 0;
+            for (int it = 0; ok; ++it) {
+                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
+                const int tile = sched_slot[ss];
+                mbar_arrive(sempty_bar(ss));
+                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+                if (tile < 0) break;
+                int mt, nt;
+                decode_tile(p, tile, mt, nt);
+                const uint32_t idesc = make_idesc(tile_n(nt), A_MN, B_MN);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
@@ -569,7 +596,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         // K-major: 16 elements = 32 B along the swizzled row; MN-major: 16 K-rows = 2048 B
                         const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
                         const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        umma_f16(tmem_d, adesc + aoff, bdesc + boff, IDESC, (kb | k) != 0 ? 1u : 0u);
+                        umma_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(empty_bar(stage));                      // frees the stage once these MMAs retire
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -586,10 +613,21 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---------------------------------------------------------------- epilogue warps
         const int quad = warp & 3;                                     // TMEM lane quadrant this warp may read
         const int row = quad * 32 + lane;
-        int it = 0; bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+        int ss = 0; uint32_t sphase = 0;
+        bool ok = true;
+        for (int it = 0; ok; ++it) {
+            int tile = -2;
+            if (lane == 0) {
+                if (mbar_wait(sfull_bar(ss), sphase, abort_flag)) {
+                    tile = sched_slot[ss];
+                    mbar_arrive(sempty_bar(ss));
+                }
+            }
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+            if (tile < 0) break;                                        // -1: no tiles left, -2: gave up
             int mt, nt;
-                decode_tile(p, tile, mt, nt);
+            decode_tile(p, tile, mt, nt);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
             if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
@@ -597,8 +635,8 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row);
-            else epilogue_dw<BN>(p, mt, nt, row, tmem_row);
+            else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
+            else epilogue_dw<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(ab));
@@ -706,8 +744,25 @@ std::mutex g_prof_mu;
 bool g_prof_on = false;
 std::vector<ProfEntry> g_prof;
 
+// Tile counters of the dynamic scheduler: one per launch, zeroed in bulk; a call that needs more
+// launches than counters zeroes them again when it wraps (stream order makes that safe).
+constexpr int NUM_TILE_COUNTERS = 1024;
+struct CounterPool {
+    int* base; int next; cudaStream_t st; bool failed;
+    CounterPool(int* b, cudaStream_t s) : base(b), next(0), st(s), failed(false) {
+        failed = cudaMemsetAsync(base, 0, 4 * NUM_TILE_COUNTERS, st) != cudaSuccess;
+    }
+    int* take() {
+        if (next == NUM_TILE_COUNTERS) {
+            failed = failed || cudaMemsetAsync(base, 0, 4 * NUM_TILE_COUNTERS, st) != cudaSuccess;
+            next = 0;
+        }
+        return base + next++;
+    }
+};
+
 struct WsLayout {
-    size_t status, scalars, sm, sz, ylab, pm, pz, G, acc, total;
+    size_t status, scalars, counters, sm, sz, ylab, pm, pz, G, acc, total;
 };
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -719,6 +774,7 @@ bool ws_layout(int64_t T_chunk, int64_t d, int64_t block_v, WsLayout* L) {
     size_t off = 0;
     L->status = off;  off += 256;
     L->scalars = off; off += 256;
+    L->counters = off; off += 4 * NUM_TILE_COUNTERS;
     L->sm = off;      off = align_up(off + 4 * T_chunk, 1024);
     L->sz = off;      off = align_up(off + 4 * T_chunk, 1024);
     L->ylab = off;    off = align_up(off + 4 * T_chunk, 1024);
@@ -820,16 +876,13 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     return cudaGetLastError();
 }
 
-// Output-column tile for the two gradient GEMMs: the widest of {256, 192, 128, 64} that wastes
-// the fewest padded columns of d.
+// Output-column tile for the two gradient GEMMs: 256 unless d is narrower; the last tile of a
+// row runs with its own (narrower) MMA width, so d need not be a multiple of the tile.
 int pick_bn(int64_t d) {
-    const int cands[4] = {256, 192, 128, 64};
-    int best = 256; int64_t best_pad = -1;
-    for (int c : cands) {
-        const int64_t pad = (d + c - 1) / c * c;
-        if (best_pad < 0 || pad < best_pad) { best = c; best_pad = pad; }
-    }
-    return best;
+    if (d <= 64) return 64;
+    if (d <= 128) return 128;
+    if (d <= 192) return 192;
+    return 256;
 }
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -922,6 +975,7 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
 
     vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
 
     const int64_t P = (V + block_v - 1) / block_v;
     const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
@@ -948,6 +1002,7 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
             p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
             p.status = status;
             apply_tuning(p, EPI_FOLD);
+            p.tile_counter = counters.take();
             if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, tmH, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
                                                                   rows, i == 0, i == P - 1, labels + tok0, ignore_index,
@@ -956,7 +1011,7 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
             if (cudaGetLastError() != cudaSuccess) return VPCE_CUDA_ERROR;
         }
     }
-    return VPCE_OK;
+    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
 }
 
 vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse, const float* dloss,
@@ -984,6 +1039,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
 
     vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
     if (!dloss) {
         vpce_count_valid_kernel<<<1, 1024, 0, st>>>(labels, T, static_cast<int>(V), ignore_index, inv_n, nullptr, status);
         g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -1022,6 +1078,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             p.G = G; p.g_ld = static_cast<int>(block_v);
             p.status = status;
             apply_tuning(p, EPI_RESID);
+            p.tile_counter = counters.take();
             if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, tmG_st, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             const int k_cols = strip_tiles_n * BN_VOCAB;               // columns of G written by step (1)
             const int m_rows = p.m_tiles * BM;                         // rows of G written by step (1)
@@ -1040,6 +1097,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             ph.status = status;
             ph.b_3d = mn3d;
             apply_tuning(ph, EPI_DH);
+            ph.tile_counter = counters.take();
             if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             // (3) dW_q += G^T H_c : M = shard vocabulary, N = d, K = chunk tokens
             GemmParams pw{};
@@ -1055,6 +1113,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             pw.status = status;
             pw.a_3d = mn3d; pw.b_3d = mn3d;
             apply_tuning(pw, EPI_DW);
+            pw.tile_counter = counters.take();
             if (launch_grad<true, true, EPI_DW>(bn, tmG_mn, tmH_mn, pw, st) != cudaSuccess) return VPCE_CUDA_ERROR;
         }
     }
@@ -1200,6 +1259,7 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
     // fully rewritten before they are read.
     vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);   // a memset, not an allocation
 
     const int64_t P = (V + block_v - 1) / block_v;
     const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
@@ -1225,6 +1285,7 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
             p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
             p.status = status;
             apply_tuning(p, EPI_FOLD);
+            p.tile_counter = counters.take();
             const int tiles = p.m_tiles * p.n_tiles;
             const int grid = tiles < num_sms() ? tiles : num_sms();
             kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmH, tmW, tmH, p);
