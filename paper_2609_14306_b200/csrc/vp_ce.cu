@@ -66,6 +66,7 @@ struct GemmParams {
     int part_ld;
     __nv_bfloat16* G;                      // [T_chunk][g_ld]
     int g_ld;
+    int g_rows;                            // rows of the G workspace (T_chunk)
     // DH
     float* acc;                            // [T_chunk][acc_ld] fp32 running dH of the chunk
     int acc_ld;
@@ -141,6 +142,87 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+// ---- cluster / CTA-pair (cta_group::2) primitives
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+    }
+}
+// TMA loads of a CTA pair: data lands in the executing CTA, the byte count is credited to `bar`,
+// which may live in the peer CTA (shared::cluster address).  No multicast.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                             uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tmem2_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem2_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem2_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma2_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma2_commit_local(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Arrives (once the issuing thread's MMAs retire) on the barrier at this offset in both CTAs of the pair.
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+}
+
 __device__ __forceinline__ uint64_t make_policy(int kind) {
     uint64_t pol;
     if (kind == 1) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -229,10 +311,10 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
     return d;
 }
 // Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = 128, N = bn.
-__host__ __device__ constexpr uint32_t make_idesc(int bn, bool a_mn, bool b_mn) {
+__host__ __device__ constexpr uint32_t make_idesc(int bn, bool a_mn, bool b_mn, int m = BM) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn) << 15) |
            (static_cast<uint32_t>(b_mn) << 16) | (static_cast<uint32_t>(bn >> 3) << 17) |
-           (static_cast<uint32_t>(BM >> 4) << 24);
+           (static_cast<uint32_t>(m >> 4) << 24);
 }
 
 template <int BN> struct StageCfg {
@@ -360,7 +442,7 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtens
         }
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) {
+        if (lane == 0 && mt * BM < p.g_rows) {                          // tiles past the workspace rows store nothing
             if (p.hint_c) tma_store_2d_hint(tmG, buf, nt * BN_VOCAB + h * 64, mt * BM + (row - lane), pol_c);
             else tma_store_2d(tmG, buf, nt * BN_VOCAB + h * 64, mt * BM + (row - lane));
             bulk_commit();
@@ -654,6 +736,207 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
+// ------------------------------------------------------------------------------------ the CTA-pair GEMM kernel
+// Two CTAs of a cluster (one TPC) work on one 256 x BN tile with tcgen05.mma.cta_group::2: each
+// CTA loads its own 128 rows of A and HALF of the B tile (BN/2 rows), the leader CTA (cluster rank
+// 0) issues the MMAs, which read both CTAs' shared memory and write both CTAs' tensor memory, and
+// each CTA drains its own 128 accumulator rows.  Per CTA and k-block this moves 16 KB + BN*64 B
+// from L2 instead of 16 KB + BN*128 B: a third less L2->SM traffic at BN = 256.
+// Signalling: TMA byte counts of both CTAs are credited to the leader's "full" barrier
+// (.cta_group::2 loads, no multicast); tcgen05.commit with a CTA mask releases the stage in both
+// CTAs and publishes the accumulator to both epilogues; epilogue warps of both CTAs arrive on the
+// leader's "accumulator free" barrier.  Tiles are assigned round-robin to the pairs.
+template <int BN> struct PairCfg {
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = (BN / 2) * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
+    static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
+};
+template <int BN, int EPI> constexpr int pair_smem_total() {
+    return PairCfg<BN>::SMEM_TOTAL + (EPI == 1 ? G_STAGING_BYTES : 0);
+}
+
+template <int BN, bool A_MN, bool B_MN, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
+    using Cfg = PairCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr uint32_t TMEM_COLS = 512u;
+    constexpr uint32_t ACC_STRIDE = 256u;
+    static_assert(BN == 256 || BN == 128, "pair tiles are 256 x 256 or 256 x 128");
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t bars = base + STAGES * Cfg::STAGE_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };                    // used in the leader only
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };   // used in the leader only
+    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const uint32_t g_staging = base + STAGES * Cfg::STAGE_BYTES + 1024;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int pair = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+    const int pm_tiles = (p.m_tiles + 1) >> 1;                               // 256-row tiles
+    const int total_tiles = pm_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem2_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem2_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                                      // the peer's barriers exist before any remote signal
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // MMA width of n-tile nt.  Each CTA supplies N/2 columns of B: N/2 must be a multiple of 16, and
+    // of 64 (one swizzled chunk) when B is MN-major.
+    auto tile_n = [&](int nt) {
+        const int left = p.cols_valid - nt * BN;
+        constexpr int R = B_MN ? 128 : 32;
+        return left >= BN ? BN : ((left + R - 1) / R * R);
+    };
+    auto decode_pair = [&](int tile, int& pmt, int& nt) {
+        const int per_group = p.group_n * pm_tiles;
+        const int g = tile / per_group;
+        const int r = tile - g * per_group;
+        const int n0 = g * p.group_n;
+        const int gw = min(p.group_n, p.n_tiles - n0);
+        pmt = r / gw;
+        nt = n0 + (r - pmt * gw);
+    };
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer (both CTAs)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            long issued = 0;
+            const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
+            for (int tile = pair; ok && tile < total_tiles; tile += num_pairs) {
+                int pmt, nt;
+                decode_pair(tile, pmt, nt);
+                const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
+                const int bn0 = nt * BN + static_cast<int>(rank) * (tile_n(nt) / 2);   // this CTA's half of the B tile
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
+                    const uint32_t bar = mapa_shared(full_bar(stage), 0);    // the leader's barrier
+                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+                    if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BK, (p.a_mn0 + mt * BM) >> 6, pol_a);
+                    else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BK, p.a_mn0 + mt * BM, pol_a);
+                    if (B_MN) tma2_load_3d(sb, &tmB, bar, 0, p.b_k0 + kb * BK, (p.b_mn0 + bn0) >> 6, pol_b);
+                    else tma2_load_2d(sb, &tmB, bar, p.b_k0 + kb * BK, p.b_mn0 + bn0, pol_b);
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if ((!ok || *abort_flag) && leader) {
+                // Give-up path (the leader's barriers count both CTAs' bytes): let copies in flight land.
+                const long back = issued < STAGES ? issued : STAGES;
+                int s = stage; uint32_t ph = phase;
+                for (long i = 0; i < back; ++i) {
+                    if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
+                    unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            int it = 0;
+            for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++it) {
+                int pmt, nt;
+                decode_pair(tile, pmt, nt);
+                const uint32_t idesc = make_idesc(tile_n(nt), A_MN, B_MN, 2 * BM);
+                const int ab = it & 1;
+                const uint32_t aphase = (it >> 1) & 1u;
+                if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+                    const uint64_t adesc = A_MN ? make_smem_desc(sa, BK * 128, 1024) : make_smem_desc(sa, 16, 1024);
+                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, BK * 128, 1024) : make_smem_desc(sb, 16, 1024);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
+                        const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
+                        umma2_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma2_commit_both(empty_bar(stage));                     // frees the stage in both CTAs
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma2_commit_both(tfull_bar(ab));                    // accumulator ready in both CTAs
+            }
+            if (!ok || *abort_flag) {
+                umma2_commit_local(drain_bar);
+                unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps (both CTAs)
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        int it = 0; bool ok = true;
+        for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++it) {
+            int pmt, nt;
+            decode_pair(tile, pmt, nt);
+            const int mt = 2 * pmt + static_cast<int>(rank);
+            const int ab = it & 1;
+            const uint32_t aphase = (it >> 1) & 1u;
+            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
+            if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
+            else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
+            else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
+            else epilogue_dw<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
+        }
+        if (EPI == EPI_RESID && lane == 0) bulk_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                          // no CTA leaves while its pair may still signal it or read its memory
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, VPCE_DEV_WAIT_EXPIRED);
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem2_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
 // ------------------------------------------------------------------------------------ small kernels
 // Folds the per-tile partial states of one strip into the running per-token state (Eq. 2
 // applied to two states: m = max(m1, m2), z = z1 e^{m1-m} + z2 e^{m2-m}), in tile order so the
@@ -876,6 +1159,48 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     return cudaGetLastError();
 }
 
+template <int BN, bool A_MN, bool B_MN, int EPI>
+cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const GemmParams& p,
+                        cudaStream_t st) {
+    constexpr int SMEM = pair_smem_total<BN, EPI>();
+    auto kern = vpce_gemm_pair_kernel<BN, A_MN, B_MN, EPI>;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const int tiles = ((p.m_tiles + 1) / 2) * p.n_tiles;
+    if (tiles <= 0 || p.num_kb <= 0) return cudaSuccess;
+    const int max_pairs = num_sms() / 2;
+    const int grid = 2 * (tiles < max_pairs ? tiles : max_pairs);
+    ProfEntry pe{EPI, nullptr, nullptr};
+    bool prof = false;
+    {
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        prof = g_prof_on;
+    }
+    if (prof && cudaEventCreate(&pe.a) == cudaSuccess && cudaEventCreate(&pe.b) == cudaSuccess) cudaEventRecord(pe.a, st);
+    else prof = false;
+    kern<<<grid, NUM_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
+    if (prof) {
+        cudaEventRecord(pe.b, st);
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        g_prof.push_back(pe);
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+// Which GEMMs run as CTA pairs (bit 0 strip kernels, bit 1 input-gradient, bit 2 weight-gradient).
+// All of them by default; VPCE_PAIR in the environment overrides it for A/B measurements.
+int pair_mask() {
+    const char* e = getenv("VPCE_PAIR");
+    return e ? atoi(e) : 7;
+}
+
 // Output-column tile for the two gradient GEMMs: 256 unless d is narrower; the last tile of a
 // row runs with its own (narrower) MMA width, so d need not be a multiple of the tile.
 int pick_bn(int64_t d) {
@@ -911,8 +1236,6 @@ void apply_tuning(GemmParams& p, int epi) {
     p.hint_a = 0;
     p.hint_b = 2;
     p.hint_c = (epi == EPI_RESID) ? 1 : 0;
-    const char* e = getenv("VPCE_HINTS");
-    if (e) { int hv = atoi(e); p.hint_a = hv / 100; p.hint_b = (hv / 10) % 10; p.hint_c = hv % 10; }
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -970,8 +1293,11 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
     float* pm = reinterpret_cast<float*>(ws + L.pm);
     float* pz = reinterpret_cast<float*>(ws + L.pz);
 
-    CUtensorMap tmH, tmW;
-    if (!make_map(&tmH, H, T, d, d, BK, BM) || !make_map(&tmW, W, V, d, d, BK, BN_VOCAB)) return VPCE_CUDA_ERROR;
+    CUtensorMap tmH, tmW, tmW_half;
+    if (!make_map(&tmH, H, T, d, d, BK, BM) || !make_map(&tmW, W, V, d, d, BK, BN_VOCAB) ||
+        !make_map(&tmW_half, W, V, d, d, BK, BN_VOCAB / 2))
+        return VPCE_CUDA_ERROR;
+    const bool pair_strip = (pair_mask() & 1) != 0;
 
     vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -1003,7 +1329,11 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
             p.status = status;
             apply_tuning(p, EPI_FOLD);
             p.tile_counter = counters.take();
-            if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, tmH, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            if (pair_strip && p.m_tiles >= 2) {
+                if (launch_pair<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW_half, tmH, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            } else if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, tmH, p, st) != cudaSuccess) {
+                return VPCE_CUDA_ERROR;
+            }
             vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
                                                                   rows, i == 0, i == P - 1, labels + tok0, ignore_index,
                                                                   static_cast<int>(V), lse + tok0, loss + tok0, status);
@@ -1046,6 +1376,12 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
     }
 
     const int bn = pick_bn(d);
+    // CTA-pair variants: half-width B boxes
+    const int pmask = pair_mask();
+    CUtensorMap tmW_khalf, tmW_mn2, tmH_mn2;
+    const bool pair_ok = (bn == 256) && (d % 64 == 0);
+    if (!make_map(&tmW_khalf, W, V, d, d, BK, BN_VOCAB / 2)) return VPCE_CUDA_ERROR;
+    if (pair_ok && (!make_map_mn3d(&tmW_mn2, W, V, d, d, 2) || !make_map_mn3d(&tmH_mn2, H, T, d, d, 2))) return VPCE_CUDA_ERROR;
     // one-instruction fetch of MN-major operands when the contiguous extent is a multiple of 64
     const bool mn3d = (d % 64 == 0);
     if (mn3d) {
@@ -1075,11 +1411,15 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             p.v_lo = static_cast<int>(v_lo);
             p.labels = labels + tok0; p.lse = lse + tok0; p.dloss = dloss ? dloss + tok0 : nullptr;
             p.inv_n_valid = inv_n; p.ignore_index = ignore_index; p.V = static_cast<int>(V);
-            p.G = G; p.g_ld = static_cast<int>(block_v);
+            p.G = G; p.g_ld = static_cast<int>(block_v); p.g_rows = static_cast<int>(T_chunk);
             p.status = status;
             apply_tuning(p, EPI_RESID);
             p.tile_counter = counters.take();
-            if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, tmG_st, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            if ((pmask & 1) && p.m_tiles >= 2) {
+                if (launch_pair<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_khalf, tmG_st, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            } else if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, tmG_st, p, st) != cudaSuccess) {
+                return VPCE_CUDA_ERROR;
+            }
             const int k_cols = strip_tiles_n * BN_VOCAB;               // columns of G written by step (1)
             const int m_rows = p.m_tiles * BM;                         // rows of G written by step (1)
             // (2) dH_c += G W_q : M = tokens, N = d, K = shard vocabulary
@@ -1098,7 +1438,11 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             ph.b_3d = mn3d;
             apply_tuning(ph, EPI_DH);
             ph.tile_counter = counters.take();
-            if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            if ((pmask & 2) && pair_ok && ph.m_tiles >= 2) {
+                if (launch_pair<256, false, true, EPI_DH>(tmG_k, tmW_mn2, tmG_k, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            } else if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) {
+                return VPCE_CUDA_ERROR;
+            }
             // (3) dW_q += G^T H_c : M = shard vocabulary, N = d, K = chunk tokens
             GemmParams pw{};
             pw.m_tiles = (cols + BM - 1) / BM;
@@ -1114,7 +1458,11 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             pw.a_3d = mn3d; pw.b_3d = mn3d;
             apply_tuning(pw, EPI_DW);
             pw.tile_counter = counters.take();
-            if (launch_grad<true, true, EPI_DW>(bn, tmG_mn, tmH_mn, pw, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            if ((pmask & 4) && pair_ok && pw.m_tiles >= 2) {
+                if (launch_pair<256, true, true, EPI_DW>(tmG_mn, tmH_mn2, tmG_mn, pw, st) != cudaSuccess) return VPCE_CUDA_ERROR;
+            } else if (launch_grad<true, true, EPI_DW>(bn, tmG_mn, tmH_mn, pw, st) != cudaSuccess) {
+                return VPCE_CUDA_ERROR;
+            }
         }
     }
     return VPCE_OK;
