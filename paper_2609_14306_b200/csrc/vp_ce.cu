@@ -1,6 +1,6 @@
 // Fused vocabulary projection + cross-entropy for sm_100a (B200).
 //
-// One warp-specialised, persistent tcgen05 GEMM kernel is instantiated with four epilogues:
+// A warp-specialised, persistent tcgen05 GEMM kernel is instantiated with four epilogues:
 //   FOLD   strip Y = H_c W_q^T  -> per-tile partial (max, sum-exp) + target logit   (Eq. 2)
 //   RESID  the same strip       -> G = dloss (exp(Y - lse) - onehot) as bf16       (App. C)
 //   DH     dH_c += G W_q        (contract over the shard's vocabulary)
@@ -8,6 +8,12 @@
 // Operands reach shared memory by TMA (128-byte swizzle), accumulators live in tensor
 // memory (two buffers, so the epilogue of tile i overlaps the MMAs of tile i+1), and the
 // logit strip never reaches global memory.
+//
+// Two variants of the kernel exist:
+//   vpce_gemm_pair_kernel  two CTAs of a cluster share one 256 x 256 tile (tcgen05 cta_group::2);
+//                          the default whenever a launch has at least two 128-row tiles;
+//   vpce_gemm_kernel       one CTA per 128 x BN tile, tiles handed out by an atomic counter;
+//                          used for narrow problems and by vp_ce_forward_static.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
 // warps 2..5 = epilogue (one thread per accumulator row).
@@ -450,8 +456,8 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtens
     }
 }
 
-template <int BN>
-__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row, int n_this) {
+// ncol0: first output column of the tile; n_this: its width (columns beyond cols_valid are skipped).
+__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
     const int grow = mt * BM + row;
     const bool row_ok = grow < p.rows_valid;
 #pragma unroll 1
@@ -460,7 +466,7 @@ __device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt,
         __syncwarp();
         tmem_ld32(tmem_row + c * 32, v);
         tmem_ld_wait();
-        const int col0 = nt * BN + c * 32;
+        const int col0 = ncol0 + c * 32;
         if (row_ok) {
         float* arow = p.acc + static_cast<size_t>(grow) * p.acc_ld + col0;
         __nv_bfloat16* orow = p.dH + static_cast<size_t>(grow) * p.out_ld + col0;
@@ -488,8 +494,7 @@ __device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nt,
     }
 }
 
-template <int BN>
-__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row, int n_this) {
+__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
     const int grow = mt * BM + row;                                    // vocabulary row within the shard
     const bool row_ok = grow < p.rows_valid;
 #pragma unroll 1
@@ -498,7 +503,7 @@ __device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nt,
         __syncwarp();
         tmem_ld32(tmem_row + c * 32, v);
         tmem_ld_wait();
-        const int col0 = nt * BN + c * 32;
+        const int col0 = ncol0 + c * 32;
         if (row_ok) {
         float* orow = p.dW + static_cast<size_t>(grow) * p.out_ld + col0;
 #pragma unroll
@@ -717,8 +722,8 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
-            else epilogue_dw<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
+            else if (EPI == EPI_DH) epilogue_dh(p, mt, nt * BN, row, tmem_row, tile_n(nt));
+            else epilogue_dw(p, mt, nt * BN, row, tmem_row, tile_n(nt));
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(ab));
@@ -817,6 +822,14 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         constexpr int R = B_MN ? 128 : 32;
         return left >= BN ? BN : ((left + R - 1) / R * R);
     };
+    // Tile list of this launch.  The first `full` entries are whole 256 x BN tiles (as many complete
+    // rounds over the pairs as there are); when the remainder would leave more than half of the pairs
+    // idle in a last round, the two gradient GEMMs cut each remaining tile into two halves of BN/2
+    // columns, so the last round costs half a tile time.
+    const int full_tiles = (EPI == EPI_DH || EPI == EPI_DW) ? (total_tiles / num_pairs) * num_pairs : total_tiles;
+    const int rem_tiles = total_tiles - full_tiles;
+    const bool split_rem = rem_tiles > 0 && 2 * rem_tiles <= num_pairs && BN == 256;
+    const int list_len = split_rem ? full_tiles + 2 * rem_tiles : total_tiles;
     auto decode_pair = [&](int tile, int& pmt, int& nt) {
         const int per_group = p.group_n * pm_tiles;
         const int g = tile / per_group;
@@ -826,6 +839,20 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         pmt = r / gw;
         nt = n0 + (r - pmt * gw);
     };
+    // Entry t of the list: 256-row tile pmt, columns [ncol0, ncol0 + width) of n-tile nt; width == 0 means "nothing".
+    auto get_tile = [&](int t, int& pmt, int& nt, int& ncol0, int& width) {
+        if (!split_rem || t < full_tiles) {
+            decode_pair(t, pmt, nt);
+            ncol0 = nt * BN;
+            width = tile_n(nt);
+            return;
+        }
+        const int v = t - full_tiles;
+        decode_pair(full_tiles + (v >> 1), pmt, nt);
+        const int w = tile_n(nt);
+        if (w <= BN / 2) { ncol0 = nt * BN; width = (v & 1) ? 0 : w; }
+        else { ncol0 = nt * BN + (v & 1) * (BN / 2); width = (v & 1) ? w - BN / 2 : BN / 2; }
+    };
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (both CTAs)
@@ -833,11 +860,12 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int stage = 0; uint32_t phase = 0; bool ok = true;
             long issued = 0;
             const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
-            for (int tile = pair; ok && tile < total_tiles; tile += num_pairs) {
-                int pmt, nt;
-                decode_pair(tile, pmt, nt);
+            for (int tile = pair; ok && tile < list_len; tile += num_pairs) {
+                int pmt, nt, ncol0, width;
+                get_tile(tile, pmt, nt, ncol0, width);
+                if (width == 0) continue;
                 const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
-                const int bn0 = nt * BN + static_cast<int>(rank) * (tile_n(nt) / 2);   // this CTA's half of the B tile
+                const int bn0 = ncol0 + static_cast<int>(rank) * (width / 2);   // this CTA's half of the B tile
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
@@ -868,10 +896,11 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         if (lane == 0 && leader) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             int it = 0;
-            for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++it) {
-                int pmt, nt;
-                decode_pair(tile, pmt, nt);
-                const uint32_t idesc = make_idesc(tile_n(nt), A_MN, B_MN, 2 * BM);
+            for (int tile = pair; ok && tile < list_len; tile += num_pairs) {
+                int pmt, nt, ncol0, width;
+                get_tile(tile, pmt, nt, ncol0, width);
+                if (width == 0) continue;
+                const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
                 if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
@@ -894,6 +923,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (ok) umma2_commit_both(tfull_bar(ab));                    // accumulator ready in both CTAs
+                ++it;
             }
             if (!ok || *abort_flag) {
                 umma2_commit_local(drain_bar);
@@ -906,9 +936,10 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         int it = 0; bool ok = true;
-        for (int tile = pair; ok && tile < total_tiles; tile += num_pairs, ++it) {
-            int pmt, nt;
-            decode_pair(tile, pmt, nt);
+        for (int tile = pair; ok && tile < list_len; tile += num_pairs) {
+            int pmt, nt, ncol0, width;
+            get_tile(tile, pmt, nt, ncol0, width);
+            if (width == 0) continue;
             const int mt = 2 * pmt + static_cast<int>(rank);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
@@ -917,11 +948,12 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
-            else epilogue_dw<BN>(p, mt, nt, row, tmem_row, tile_n(nt));
+            else if (EPI == EPI_DH) epilogue_dh(p, mt, ncol0, row, tmem_row, width);
+            else epilogue_dw(p, mt, ncol0, row, tmem_row, width);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
+            ++it;
         }
         if (EPI == EPI_RESID && lane == 0) bulk_wait_all();
     }
