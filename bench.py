@@ -91,9 +91,11 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample_rate(w, W_bits, H_bits, labels, budget_s=15.0):
+def oracle_sample_rate(w, W_bits, H_bits, labels, n_tokens=1024, W64=None):
     """Times the float64 oracle (as it stands) on the first n tokens of the batch against the whole
-    vocabulary; n is sized from a short probe so that the timed call takes about `budget_s`."""
+    vocabulary.  The oracle works through token slabs of 1024 rows and pays O(V d) per slab for its
+    float64 dW accumulation, so one full slab is the smallest sample with the steady-state cost of a
+    whole run; smaller samples overstate the per-token cost."""
     from oracle import vpce_oracle as orc
     from synth_inputs import IGNORE_INDEX, bf16_bits_to_f64
     try:
@@ -101,14 +103,9 @@ def oracle_sample_rate(w, W_bits, H_bits, labels, budget_s=15.0):
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
     except Exception:
         cores = os.cpu_count() or 1
-    W64 = bf16_bits_to_f64(W_bits)
-    probe = min(32, w.T)
-    t0 = time.perf_counter()
-    orc.forward_backward(bf16_bits_to_f64(H_bits[:probe]), W64, labels[:probe], None, IGNORE_INDEX)
-    per_tok = (time.perf_counter() - t0) / probe
-    n = int(max(probe, min(w.T, budget_s / max(per_tok, 1e-9))))
-    n = max(32, (n // 32) * 32) if w.T >= 32 else w.T
-    n = min(n, w.T)
+    if W64 is None:
+        W64 = bf16_bits_to_f64(W_bits)                    # input preparation, outside the timed call
+    n = min(int(n_tokens), w.T)
     t0 = time.perf_counter()
     orc.forward_backward(bf16_bits_to_f64(H_bits[:n]), W64, labels[:n], None, IGNORE_INDEX)
     dt = time.perf_counter() - t0
@@ -127,11 +124,14 @@ def run_reference(args, w):
     labels = stream_labels(w)[:w.T]
     H_bits = make_hidden(w, 0)
     steps = max(1, args.steps)
-    budget = max(2.0, min(15.0, 120.0 / (steps + args.warmup)))
+    # one oracle slab (1024 tokens) per step when the run is short, fewer tokens per step when K + W is large
+    n_step = max(256, min(1024, (1024 * 6 // (steps + args.warmup)) // 32 * 32))
+    from synth_inputs import bf16_bits_to_f64
+    W64 = bf16_bits_to_f64(W_bits)
     res, n, dt = None, 0, 0.0
     times = []
     for i in range(args.warmup + steps):
-        res, n, dt = oracle_sample_rate(w, W_bits, H_bits, labels, budget_s=budget)
+        res, n, dt = oracle_sample_rate(w, W_bits, H_bits, labels, n_tokens=n_step, W64=W64)
         if i >= args.warmup:
             times.append(dt)
     ms = 1e3 * sum(times) / len(times)
