@@ -28,6 +28,8 @@
  *     errors only; conditions found on the device (a label outside [0, V) that is not
  *     ignore_index; a bounded wait inside a kernel that ran out) set a status word in the
  *     workspace, read back with vp_ce_device_status.
+ *   - T == 0 (an empty batch) is accepted by vp_ce_forward and vp_ce_backward: nothing is launched;
+ *     the backward zeroes dW when accumulate_dW == 0.  Other non-positive sizes are VPCE_INVALID_ARG.
  *   - A token whose label equals ignore_index has loss 0 and a zero gradient row; its lse
  *     is still computed.  A label outside [0, V) is treated the same way and flagged.
  */

@@ -1313,6 +1313,7 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
                           int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
                           int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream) {
     WsLayout L;
+    if (T == 0) return VPCE_OK;                                        // empty batch: nothing to compute
     if (!loss || !lse) return VPCE_INVALID_ARG;
     vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
     if (s != VPCE_OK) return s;
@@ -1381,6 +1382,12 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
                            int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW, void* workspace,
                            size_t workspace_bytes, void* stream) {
     WsLayout L;
+    if (T == 0) {                                                      // empty batch: dW gets no contribution
+        if (!accumulate_dW && dW && V > 0 && d > 0 &&
+            cudaMemsetAsync(dW, 0, static_cast<size_t>(V) * d * 4, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return VPCE_CUDA_ERROR;
+        return VPCE_OK;
+    }
     if (!lse || !dH || !dW) return VPCE_INVALID_ARG;
     vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
     if (s != VPCE_OK) return s;

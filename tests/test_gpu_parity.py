@@ -167,3 +167,45 @@ def test_host_side_argument_checks():
     with pytest.raises(vp.VpceError) as ei:
         vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, -1, r.ws)
     assert ei.value.code == 1
+
+
+@pytest.mark.parametrize("T,d,V,block_v,T_chunk", [
+    (1, 8, 1, 256, 128),          # a single token, a single class: loss 0
+    (5, 16, 3, 256, 128),         # everything smaller than one tile
+    (130, 72, 257, 256, 128),     # one row past a tile, one column past a vocabulary tile
+    (256, 8, 512, 256, 256),      # the narrowest hidden width the layout rules allow
+])
+def test_degenerate_small_shapes(T, d, V, block_v, T_chunk):
+    w = custom_workload(f"s{T}x{d}x{V}", T=T, d=d, V=V, block_v=block_v, T_chunk=T_chunk, w_std=0.3,
+                        labels="uniform", ignore_frac=0.0, seed=T * 7 + V)
+    b = make_batch(w)
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    run = GpuRun(b.H_bits, b.W_bits, b.labels, block_v, T_chunk).forward().backward()
+    assert run.fwd_status == 0 and run.bwd_status == 0
+    ref = orc.forward_backward(H64, W64, b.labels)
+    assert np.abs(run.np_lse() - ref["lse"]).max() <= TOL_TOKEN
+    assert np.abs(run.np_loss() - ref["loss"]).max() <= TOL_TOKEN
+    if V == 1:
+        assert not run.np_loss().any()
+        assert np.abs(run.np_dH()).max() < 1e-6 and np.abs(run.np_dW()).max() < 1e-6
+    else:
+        assert relF(run.np_dH(), ref["dH"]) <= TOL_GRAD and relF(run.np_dW(), ref["dW"]) <= TOL_GRAD
+
+
+def test_empty_batch_is_a_no_op():
+    w = custom_workload("empty", T=128, d=64, V=512, block_v=256, T_chunk=128, seed=3)
+    b = make_batch(w)
+    r = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
+    H0 = r.H[:0].contiguous()
+    lab0 = r.labels[:0].contiguous()
+    out0 = torch.empty(0, dtype=torch.float32, device="cuda")
+    vp.vp_ce_forward(H0, r.W, lab0, w.block_v, IGNORE_INDEX, out0, out0, w.T_chunk, 0, r.ws)
+    dW = torch.full((w.V, w.d), 7.0, dtype=torch.float32, device="cuda")
+    vp.vp_ce_backward(H0, r.W, lab0, out0, None, torch.empty(0, w.d, dtype=torch.bfloat16, device="cuda"), dW,
+                      w.block_v, IGNORE_INDEX, w.T_chunk, 0, True, r.ws)
+    torch.cuda.synchronize()
+    assert float(dW.min()) == 7.0 and float(dW.max()) == 7.0          # accumulate: untouched
+    vp.vp_ce_backward(H0, r.W, lab0, out0, None, torch.empty(0, w.d, dtype=torch.bfloat16, device="cuda"), dW,
+                      w.block_v, IGNORE_INDEX, w.T_chunk, 0, False, r.ws)
+    torch.cuda.synchronize()
+    assert not dW.any()                                                # overwrite: zero contribution
