@@ -27,6 +27,7 @@
 #include <cuda_runtime.h>
 #include <cudaTypedefs.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdint>
 #include <cstdio>
@@ -54,6 +55,7 @@ struct GemmParams {
     int m_tiles, n_tiles, num_kb;
     int a_3d, b_3d;                        // MN-major operand fetched as one 3-D box (64 x 64 x chunks) per k-block
     int hint_a, hint_b, hint_c;            // L2 eviction hints for A loads, B loads, C stores: 0 normal, 1 first, 2 last
+    int n_cut;                             // pair kernel: full-width tiles run as two halves at the end of the list
     int group_n;                           // n-tiles per raster group (tiles run m-major inside a group)
     int a_mn0, a_k0, b_mn0, b_k0;          // TMA coordinate bases (elements)
     int rows_valid;                        // valid accumulator rows overall (M bound)
@@ -770,7 +772,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     constexpr int STAGES = Cfg::STAGES;
     constexpr uint32_t TMEM_COLS = 512u;
     constexpr uint32_t ACC_STRIDE = 256u;
-    static_assert(BN == 256 || BN == 128, "pair tiles are 256 x 256 or 256 x 128");
+    static_assert(BN == 256, "pair tiles are 256 x 256");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -782,24 +784,29 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };   // used in the leader only
     const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 5));
+    auto sfull_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + s); };
+    auto sempty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + SCHED_DEPTH + s); };   // used in the leader only
+    constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * SCHED_DEPTH;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* sched_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [SCHED_DEPTH] list positions
+    const uint32_t sched_slot_addr = bars + 8u * NUM_BARS + 8u;
     const uint32_t g_staging = base + STAGES * Cfg::STAGE_BYTES + 1024;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
-    const int pair = blockIdx.x >> 1;
-    const int num_pairs = gridDim.x >> 1;
     const int pm_tiles = (p.m_tiles + 1) >> 1;                               // 256-row tiles
-    const int total_tiles = pm_tiles * p.n_tiles;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
         mbar_init(drain_bar, 1);
+        // a slot is free again when the leader's MMA lane + 4 epilogue warps and the peer's producer + 4 epilogue
+        // warps have read it: 10 arrivals on the leader's barrier
+        for (int s = 0; s < SCHED_DEPTH; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 10); }
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tensormap(&tmA);
@@ -822,48 +829,72 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         constexpr int R = B_MN ? 128 : 32;
         return left >= BN ? BN : ((left + R - 1) / R * R);
     };
-    // Tile list of this launch.  The first `full` entries are whole 256 x BN tiles (as many complete
-    // rounds over the pairs as there are); when the remainder would leave more than half of the pairs
-    // idle in a last round, the two gradient GEMMs cut each remaining tile into two halves of BN/2
-    // columns, so the last round costs half a tile time.
-    const int full_tiles = (EPI == EPI_DH || EPI == EPI_DW) ? (total_tiles / num_pairs) * num_pairs : total_tiles;
-    const int rem_tiles = total_tiles - full_tiles;
-    const bool split_rem = rem_tiles > 0 && 2 * rem_tiles <= num_pairs && BN == 256;
-    const int list_len = split_rem ? full_tiles + 2 * rem_tiles : total_tiles;
-    auto decode_pair = [&](int tile, int& pmt, int& nt) {
-        const int per_group = p.group_n * pm_tiles;
+    // The work list, longest items first, handed out dynamically (greedy list scheduling):
+    //   [0, n_whole)                  whole 256 x 256 tiles, n-fastest inside raster groups over the full-width n-tiles;
+    //   [n_whole, n_whole + 2*n_cut)  the last n_cut full-width tiles as two 128-column halves each (gradient GEMMs
+    //                                 only, and only when the host's estimate says the last round ends sooner that way);
+    //   the rest                      the narrower last n-tile of every row, when the width is not a multiple of 256.
+    constexpr bool kSplit = (EPI == EPI_DH || EPI == EPI_DW);
+    const int n_wide = p.cols_valid / BN;                                    // full-width n-tiles per row
+    const int n_wide_tiles = pm_tiles * n_wide;
+    const int n_cut = kSplit ? min(p.n_cut, n_wide_tiles) : 0;              // chosen by the host (pick_n_cut)
+    const int n_whole = n_wide_tiles - n_cut;
+    const int n_tail = (p.n_tiles > n_wide) ? pm_tiles : 0;
+    const int list_len = n_whole + 2 * n_cut + n_tail;
+    auto decode_wide = [&](int tile, int& pmt, int& nt) {                    // raster order over the full-width n-tiles
+        const int gn = min(p.group_n, max(n_wide, 1));
+        const int per_group = gn * pm_tiles;
         const int g = tile / per_group;
         const int r = tile - g * per_group;
-        const int n0 = g * p.group_n;
-        const int gw = min(p.group_n, p.n_tiles - n0);
+        const int n0 = g * gn;
+        const int gw = min(gn, n_wide - n0);
         pmt = r / gw;
         nt = n0 + (r - pmt * gw);
     };
-    // Entry t of the list: 256-row tile pmt, columns [ncol0, ncol0 + width) of n-tile nt; width == 0 means "nothing".
     auto get_tile = [&](int t, int& pmt, int& nt, int& ncol0, int& width) {
-        if (!split_rem || t < full_tiles) {
-            decode_pair(t, pmt, nt);
-            ncol0 = nt * BN;
-            width = tile_n(nt);
-            return;
+        if (t < n_whole) {
+            decode_wide(t, pmt, nt);
+            ncol0 = nt * BN; width = BN;
+        } else if (t < n_whole + 2 * n_cut) {
+            const int v = t - n_whole;
+            decode_wide(n_whole + (v >> 1), pmt, nt);
+            ncol0 = nt * BN + (v & 1) * (BN / 2); width = BN / 2;
+        } else {
+            pmt = t - (n_whole + 2 * n_cut);
+            nt = n_wide;
+            ncol0 = nt * BN; width = tile_n(nt);
         }
-        const int v = t - full_tiles;
-        decode_pair(full_tiles + (v >> 1), pmt, nt);
-        const int w = tile_n(nt);
-        if (w <= BN / 2) { ncol0 = nt * BN; width = (v & 1) ? 0 : w; }
-        else { ncol0 = nt * BN + (v & 1) * (BN / 2); width = (v & 1) ? w - BN / 2 : BN / 2; }
     };
+    // Scheduler ring: the leader's producer lane takes list positions from the launch's counter and writes them
+    // into the same slot of both CTAs; every reader acknowledges on the leader's "slot free" barrier.
+    auto sched_ack = [&](int ss) { mbar_arrive_cluster(mapa_shared(sempty_bar(ss), 0)); };
 
     if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer (both CTAs)
+        // ---------------------------------------------------------------- scheduler (leader) + TMA producer (both CTAs)
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
+            int ss = 0; uint32_t sphase = 0;
             long issued = 0;
             const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
-            for (int tile = pair; ok && tile < list_len; tile += num_pairs) {
+            while (ok) {
+                int tile;
+                if (leader) {
+                    if (!mbar_wait_cluster(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    tile = atomicAdd(p.tile_counter, 1);
+                    if (tile >= list_len) tile = -1;
+                    sched_slot[ss] = tile;
+                    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(sched_slot_addr + 4u * ss, 1)), "r"(tile) : "memory");
+                    mbar_arrive(sfull_bar(ss));
+                    mbar_arrive_cluster(mapa_shared(sfull_bar(ss), 1));      // release.cluster: the peer sees its slot
+                } else {
+                    if (!mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
+                    tile = sched_slot[ss];
+                    sched_ack(ss);
+                }
+                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+                if (tile < 0) break;
                 int pmt, nt, ncol0, width;
                 get_tile(tile, pmt, nt, ncol0, width);
-                if (width == 0) continue;
                 const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
                 const int bn0 = ncol0 + static_cast<int>(rank) * (width / 2);   // this CTA's half of the B tile
                 for (int kb = 0; kb < p.num_kb; ++kb) {
@@ -895,11 +926,15 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         // ---------------------------------------------------------------- MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            int it = 0;
-            for (int tile = pair; ok && tile < list_len; tile += num_pairs) {
+            int ss = 0; uint32_t sphase = 0;
+            for (int it = 0; ok; ++it) {
+                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
+                const int tile = sched_slot[ss];
+                sched_ack(ss);
+                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+                if (tile < 0) break;
                 int pmt, nt, ncol0, width;
                 get_tile(tile, pmt, nt, ncol0, width);
-                if (width == 0) continue;
                 const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
@@ -923,7 +958,6 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (ok) umma2_commit_both(tfull_bar(ab));                    // accumulator ready in both CTAs
-                ++it;
             }
             if (!ok || *abort_flag) {
                 umma2_commit_local(drain_bar);
@@ -935,11 +969,21 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         // ---------------------------------------------------------------- epilogue warps (both CTAs)
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
-        int it = 0; bool ok = true;
-        for (int tile = pair; ok && tile < list_len; tile += num_pairs) {
+        int ss = 0; uint32_t sphase = 0;
+        bool ok = true;
+        for (int it = 0; ok; ++it) {
+            int tile = -2;
+            if (lane == 0) {
+                if (mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) {
+                    tile = sched_slot[ss];
+                    sched_ack(ss);
+                }
+            }
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+            if (tile < 0) break;                                             // -1: list exhausted, -2: gave up
             int pmt, nt, ncol0, width;
             get_tile(tile, pmt, nt, ncol0, width);
-            if (width == 0) continue;
             const int mt = 2 * pmt + static_cast<int>(rank);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
@@ -953,7 +997,6 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
-            ++it;
         }
         if (EPI == EPI_RESID && lane == 0) bulk_wait_all();
     }
@@ -1226,6 +1269,27 @@ cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     return cudaGetLastError();
 }
 
+// How many of the full-width 256 x 256 tiles of a gradient GEMM to run as two 128-column halves.
+// After the whole rounds, R = tiles % pairs full tiles and the narrow last-column tiles are left;
+// greedy list scheduling of that remainder is simulated with and without cutting the R tiles
+// (a half costs a little more than half a tile: it re-loads A and wastes half of each B box).
+int pick_n_cut(int pm_tiles, int n_wide, int tail_width, int pairs) {
+    const int wide = pm_tiles * n_wide;
+    const int R = wide % pairs;
+    if (R == 0 || pairs <= 0) return 0;
+    const double half_cost = 0.56, tail_cost = tail_width > 0 ? 1.05 * tail_width / 256.0 : 0.0;
+    const int n_tail = tail_width > 0 ? pm_tiles : 0;
+    auto makespan = [&](int n_full, int n_half) {
+        std::vector<double> load(pairs, 0.0);
+        auto put = [&](double c) { *std::min_element(load.begin(), load.end()) += c; };
+        for (int i = 0; i < n_full; ++i) put(1.0);
+        for (int i = 0; i < n_half; ++i) put(half_cost);
+        for (int i = 0; i < n_tail; ++i) put(tail_cost);
+        return *std::max_element(load.begin(), load.end());
+    };
+    return makespan(0, 2 * R) + 0.02 < makespan(R, 0) ? R : 0;
+}
+
 // Which GEMMs run as CTA pairs (bit 0 strip kernels, bit 1 input-gradient, bit 2 weight-gradient).
 // All of them by default; VPCE_PAIR in the environment overrides it for A/B measurements.
 int pair_mask() {
@@ -1475,6 +1539,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             ph.first = (i == 0); ph.last = (i == P - 1);
             ph.status = status;
             ph.b_3d = mn3d;
+            ph.n_cut = pick_n_cut((ph.m_tiles + 1) / 2, static_cast<int>(d / 256), static_cast<int>(d % 256 ? ((d % 256 + 127) / 128 * 128) : 0), num_sms() / 2);
             apply_tuning(ph, EPI_DH);
             ph.tile_counter = counters.take();
             if ((pmask & 2) && pair_ok && ph.m_tiles >= 2) {
@@ -1495,6 +1560,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             pw.accumulate = (accumulate_dW != 0) || (c > 0);
             pw.status = status;
             pw.a_3d = mn3d; pw.b_3d = mn3d;
+            pw.n_cut = pick_n_cut((pw.m_tiles + 1) / 2, static_cast<int>(d / 256), static_cast<int>(d % 256 ? ((d % 256 + 127) / 128 * 128) : 0), num_sms() / 2);
             apply_tuning(pw, EPI_DW);
             pw.tile_counter = counters.take();
             if ((pmask & 4) && pair_ok && pw.m_tiles >= 2) {
