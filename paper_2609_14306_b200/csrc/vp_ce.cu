@@ -36,1061 +36,11 @@
 #include <vector>
 
 #include "vp_ce.h"
+#include "vp_ce_kernels.cuh"
 
 namespace {
 
-constexpr int BM = 128;          // accumulator rows per tile (TMEM lanes)
-constexpr int BK = 64;           // K elements per pipeline stage (one 128-byte swizzle row of bf16)
-constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
-constexpr int BN_VOCAB = 256;    // vocabulary columns per strip tile
-constexpr int NUM_THREADS = 192;
-constexpr int SMEM_BUDGET = 200 * 1024;    // operand stages
-constexpr int SMEM_EXTRA = 2048;           // barriers + alignment slack
-constexpr int G_STAGING_BYTES = 4 * 2 * 4096;   // RESID: per epilogue warp two 32-row x 64-column bf16 boxes
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
-
-enum Epilogue { EPI_FOLD = 0, EPI_RESID = 1, EPI_DH = 2, EPI_DW = 3 };
-
-struct GemmParams {
-    int m_tiles, n_tiles, num_kb;
-    int a_3d, b_3d;                        // MN-major operand fetched as one 3-D box (64 x 64 x chunks) per k-block
-    int hint_a, hint_b, hint_c;            // L2 eviction hints for A loads, B loads, C stores: 0 normal, 1 first, 2 last
-    int n_cut;                             // pair kernel: full-width tiles run as two halves at the end of the list
-    int group_n;                           // n-tiles per raster group (tiles run m-major inside a group)
-    int a_mn0, a_k0, b_mn0, b_k0;          // TMA coordinate bases (elements)
-    int rows_valid;                        // valid accumulator rows overall (M bound)
-    int cols_valid;                        // valid accumulator columns overall (N bound)
-    // FOLD / RESID
-    int v_lo;                              // first vocabulary id of the shard
-    const int32_t* labels;                 // chunk base
-    const float* lse;                      // chunk base
-    const float* dloss;                    // chunk base or null
-    const float* inv_n_valid;              // scalar used when dloss == null
-    int ignore_index;
-    int V;
-    float* pm;                             // [n_tile][part_ld] partial max
-    float* pz;                             // [n_tile][part_ld] partial sum-exp
-    float* ylab;                           // [part_ld] target logit
-    int part_ld;
-    __nv_bfloat16* G;                      // [T_chunk][g_ld]
-    int g_ld;
-    int g_rows;                            // rows of the G workspace (T_chunk)
-    // DH
-    float* acc;                            // [T_chunk][acc_ld] fp32 running dH of the chunk
-    int acc_ld;
-    __nv_bfloat16* dH;                     // chunk base, leading dimension out_ld
-    int first, last;
-    // DW
-    float* dW;                             // shard base (row v_lo), leading dimension out_ld
-    int accumulate;
-    int out_ld;
-    int* status;
-    int* tile_counter;                     // zero before the launch; tiles are taken with atomicAdd
-};
-
-// ------------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false when the wait ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    unsigned long long t0 = 0;
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            unsigned long long now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
-        }
-    }
-}
-__device__ __forceinline__ void fence_barrier_init() {
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-// ---- cluster / CTA-pair (cta_group::2) primitives
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    unsigned long long t0 = 0;
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            unsigned long long now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
-        }
-    }
-}
-// TMA loads of a CTA pair: data lands in the executing CTA, the byte count is credited to `bar`,
-// which may live in the peer CTA (shared::cluster address).  No multicast.
-__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                             uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%3, %4, %5}], [%2], %6;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tmem2_alloc(uint32_t dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tmem2_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem2_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma2_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma2_commit_local(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// Arrives (once the issuing thread's MMAs retire) on the barrier at this offset in both CTAs of the pair.
-__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
-}
-
-__device__ __forceinline__ uint64_t make_policy(int kind) {
-    uint64_t pol;
-    if (kind == 1) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    else if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                                 uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                                 uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%3, %4, %5}], [%2], %6;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, uint32_t src, int c0, int c1, uint64_t policy) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-    uint32_t* r = reinterpret_cast<uint32_t*>(v);
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ float ex2f(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Shared-memory matrix descriptor (sm_100 format), 128-byte swizzle.
-//   K-major operand : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (SBO); LBO unused.
-//   MN-major operand: 64 K-rows of 64 MN elements (128 B) per box; boxes of successive
-//                     64-element MN chunks LBO bytes apart; 8-K-row groups 1024 B apart (SBO).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
-    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= 1ull << 46;                      // descriptor version of sm_100
-    d |= 2ull << 61;                      // SWIZZLE_128B
-    return d;
-}
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = 128, N = bn.
-__host__ __device__ constexpr uint32_t make_idesc(int bn, bool a_mn, bool b_mn, int m = BM) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn) << 15) |
-           (static_cast<uint32_t>(b_mn) << 16) | (static_cast<uint32_t>(bn >> 3) << 17) |
-           (static_cast<uint32_t>(m >> 4) << 24);
-}
-
-template <int BN> struct StageCfg {
-    static constexpr int A_BYTES = BM * BK * 2;
-    static constexpr int B_BYTES = BN * BK * 2;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
-    static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
-    // the residual epilogue stages its bf16 tile in shared memory for TMA stores
-    static constexpr int SMEM_TOTAL_STAGED = SMEM_TOTAL + G_STAGING_BYTES;
-};
-template <int BN, int EPI> constexpr int smem_total() {
-    return EPI == 1 ? StageCfg<BN>::SMEM_TOTAL_STAGED : StageCfg<BN>::SMEM_TOTAL;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&t);
-}
-
-// Tile order: the n-tiles are cut into groups of group_n; inside a group the index runs n-fastest
-// over all m-tiles, so the group's B operand (a slice of the shard) stays in L2 while A streams.
-__device__ __forceinline__ void decode_tile(const GemmParams& p, int tile, int& mt, int& nt) {
-    const int per_group = p.group_n * p.m_tiles;
-    const int g = tile / per_group;
-    const int r = tile - g * per_group;
-    const int n0 = g * p.group_n;
-    const int gw = min(p.group_n, p.n_tiles - n0);
-    mt = r / gw;
-    nt = n0 + (r - mt * gw);
-}
-
-// ------------------------------------------------------------------------------------ epilogues
-// Each epilogue thread owns accumulator row `row` (0..127) of the tile; `tmem_row` is the
-// TMEM address of that thread's lane quadrant at the accumulator's first column.
-constexpr float LOG2E = 1.4426950408889634f;
-constexpr float NEG_INF = -__builtin_huge_valf();
-
-__device__ __forceinline__ void epilogue_fold(const GemmParams& p, int mt, int nt, int row, uint32_t tmem_row) {
-    const int grow = mt * BM + row;                             // row within the chunk
-    const bool row_ok = grow < p.rows_valid;
-    const int label = row_ok ? p.labels[grow] : -1;
-    const int lrel = label - (p.v_lo + nt * BN_VOCAB);          // target column relative to the tile
-    float m = NEG_INF, z = 0.f, yl = 0.f;
-    bool hit = false;
-#pragma unroll 1
-    for (int c = 0; c < BN_VOCAB / 32; ++c) {
-        float v[32];
-        __syncwarp();
-        tmem_ld32(tmem_row + c * 32, v);
-        tmem_ld_wait();
-        const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);     // valid columns left in the shard
-        if (nvalid < 32) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) if (j >= nvalid) v[j] = NEG_INF;
-        }
-        if (static_cast<unsigned>(lrel - c * 32) < 32u) {
-            const int jj = lrel - c * 32;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) if (j == jj) yl = v[j];
-            hit = true;
-        }
-        float cmax = v[0];
-#pragma unroll
-        for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
-        const float m_new = fmaxf(m, cmax);
-        const float mL = (m_new == NEG_INF) ? 0.f : m_new * LOG2E;
-        float s = 0.f;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) s += ex2f(fmaf(v[j], LOG2E, -mL));
-        z = z * ex2f(fmaf(m, LOG2E, -mL)) + s;                         // m = -inf gives factor 0
-        m = m_new;
-    }
-    if (row_ok) {
-        p.pm[static_cast<size_t>(nt) * p.part_ld + grow] = m;
-        p.pz[static_cast<size_t>(nt) * p.part_ld + grow] = z;
-        if (hit) p.ylab[grow] = yl;                                    // exactly one tile owns the target
-    }
-}
-
-// The bf16 residual tile leaves through shared memory: each epilogue warp owns 32 rows; per 64
-// columns it fills a 32 x 128-byte box (128-byte swizzle: 16-byte chunk j of row r sits at chunk
-// j ^ (r & 7)) and one lane issues a TMA store, so global writes are whole 128-byte lines.
-__device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtensorMap* tmG, uint32_t stage_smem,
-                                               int mt, int nt, int row, int lane, uint32_t tmem_row) {
-    const int grow = mt * BM + row;
-    const bool row_ok = grow < p.rows_valid;
-    int label = row_ok ? p.labels[grow] : p.ignore_index;
-    const bool valid = row_ok && label != p.ignore_index && static_cast<unsigned>(label) < static_cast<unsigned>(p.V);
-    float dl = 0.f, lseL = 0.f;
-    if (valid) dl = p.dloss ? p.dloss[grow] : *p.inv_n_valid;
-    if (row_ok) lseL = p.lse[grow] * LOG2E;
-    const int lrel = valid ? label - (p.v_lo + nt * BN_VOCAB) : -1;
-    const uint64_t pol_c = make_policy(p.hint_c);
-#pragma unroll 1
-    for (int h = 0; h < BN_VOCAB / 64; ++h) {
-        const uint32_t buf = stage_smem + (h & 1) * 4096;
-        if (lane == 0) bulk_wait_read_1();                              // the store that last read this buffer is done
-        __syncwarp();
-#pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-            const int c = 2 * h + c2;
-            float v[32];
-            __syncwarp();
-            tmem_ld32(tmem_row + c * 32, v);
-            tmem_ld_wait();
-            const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);
-            const int jj = lrel - c * 32;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float g = dl * ex2f(fmaf(v[j], LOG2E, -lseL));
-                if (j == jj) g -= dl;
-                v[j] = (j < nvalid) ? g : 0.f;
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint4 o;
-                o.x = pack_bf16x2(v[8 * q + 0], v[8 * q + 1]);
-                o.y = pack_bf16x2(v[8 * q + 2], v[8 * q + 3]);
-                o.z = pack_bf16x2(v[8 * q + 4], v[8 * q + 5]);
-                o.w = pack_bf16x2(v[8 * q + 6], v[8 * q + 7]);
-                const int chunk = c2 * 4 + q;                           // 16-byte chunk within the 128-byte row
-                st_shared_v4(buf + lane * 128 + ((chunk ^ (lane & 7)) << 4), o);   // rows >= rows_valid get zeros
-            }
-        }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0 && mt * BM < p.g_rows) {                          // tiles past the workspace rows store nothing
-            if (p.hint_c) tma_store_2d_hint(tmG, buf, nt * BN_VOCAB + h * 64, mt * BM + (row - lane), pol_c);
-            else tma_store_2d(tmG, buf, nt * BN_VOCAB + h * 64, mt * BM + (row - lane));
-            bulk_commit();
-        }
-    }
-}
-
-// ncol0: first output column of the tile; n_this: its width (columns beyond cols_valid are skipped).
-__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
-    const int grow = mt * BM + row;
-    const bool row_ok = grow < p.rows_valid;
-#pragma unroll 1
-    for (int c = 0; c < (n_this + 31) / 32; ++c) {
-        float v[32];
-        __syncwarp();
-        tmem_ld32(tmem_row + c * 32, v);
-        tmem_ld_wait();
-        const int col0 = ncol0 + c * 32;
-        if (row_ok) {
-        float* arow = p.acc + static_cast<size_t>(grow) * p.acc_ld + col0;
-        __nv_bfloat16* orow = p.dH + static_cast<size_t>(grow) * p.out_ld + col0;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {                                  // 8 columns per step
-            if (col0 + 8 * q >= p.cols_valid) break;                   // d is a multiple of 8
-            float* x = v + 8 * q;
-            if (!p.first) {
-                const float4 a0 = *reinterpret_cast<const float4*>(arow + 8 * q);
-                const float4 a1 = *reinterpret_cast<const float4*>(arow + 8 * q + 4);
-                x[0] += a0.x; x[1] += a0.y; x[2] += a0.z; x[3] += a0.w;
-                x[4] += a1.x; x[5] += a1.y; x[6] += a1.z; x[7] += a1.w;
-            }
-            if (p.last) {
-                uint4 o;
-                o.x = pack_bf16x2(x[0], x[1]); o.y = pack_bf16x2(x[2], x[3]);
-                o.z = pack_bf16x2(x[4], x[5]); o.w = pack_bf16x2(x[6], x[7]);
-                *reinterpret_cast<uint4*>(orow + 8 * q) = o;
-            } else {
-                *reinterpret_cast<float4*>(arow + 8 * q) = make_float4(x[0], x[1], x[2], x[3]);
-                *reinterpret_cast<float4*>(arow + 8 * q + 4) = make_float4(x[4], x[5], x[6], x[7]);
-            }
-        }
-        }
-    }
-}
-
-__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
-    const int grow = mt * BM + row;                                    // vocabulary row within the shard
-    const bool row_ok = grow < p.rows_valid;
-#pragma unroll 1
-    for (int c = 0; c < (n_this + 31) / 32; ++c) {
-        float v[32];
-        __syncwarp();
-        tmem_ld32(tmem_row + c * 32, v);
-        tmem_ld_wait();
-        const int col0 = ncol0 + c * 32;
-        if (row_ok) {
-        float* orow = p.dW + static_cast<size_t>(grow) * p.out_ld + col0;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {                                  // 4 columns per step
-            if (col0 + 4 * q >= p.cols_valid) break;
-            float4 x = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-            if (p.accumulate) {
-                const float4 a = *reinterpret_cast<const float4*>(orow + 4 * q);
-                x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
-            }
-            *reinterpret_cast<float4*>(orow + 4 * q) = x;
-        }
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------ the GEMM kernel
-// Tiles are handed out dynamically: the producer lane takes the next tile index from a global
-// counter (atomicAdd) and publishes it to the MMA lane and the epilogue warps through a small
-// shared-memory ring guarded by mbarriers, so a CTA that finishes early simply takes more tiles.
-// The last n-tile of a row may be narrower than BN (its MMA uses N = valid columns rounded up
-// to 16), so an output width that is not a multiple of BN costs no padded tensor-core work.
-constexpr int SCHED_DEPTH = 4;
-
-template <int BN, bool A_MN, bool B_MN, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-    using Cfg = StageCfg<BN>;
-    constexpr int STAGES = Cfg::STAGES;
-    constexpr uint32_t TMEM_COLS = (BN > 128) ? 512u : (BN > 64 ? 256u : 128u);
-    constexpr uint32_t ACC_STRIDE = TMEM_COLS / 2;
-
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;                      // swizzle atoms need 1024-byte alignment
-    uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t bars = base + STAGES * Cfg::STAGE_BYTES;            // 8-byte barriers after the stages
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
-    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
-    auto sfull_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + s); };
-    auto sempty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + SCHED_DEPTH + s); };
-    constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * SCHED_DEPTH;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * NUM_BARS);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* sched_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [SCHED_DEPTH] tile ids
-    const uint32_t g_staging = base + STAGES * Cfg::STAGE_BYTES + 1024;   // RESID only (1024-byte aligned)
-
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-    const int total_tiles = p.m_tiles * p.n_tiles;
-
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
-        mbar_init(drain_bar, 1);
-        for (int s = 0; s < SCHED_DEPTH; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 5); }
-        fence_barrier_init();
-        fence_proxy_async();
-        prefetch_tensormap(&tmA);
-        prefetch_tensormap(&tmB);
-    }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    // Valid accumulator columns of n-tile nt, rounded up to the MMA's granularity of 16.
-    auto tile_n = [&](int nt) {
-        const int left = p.cols_valid - nt * BN;
-        return left >= BN ? BN : ((left + 15) & ~15);
-    };
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- scheduler + TMA producer
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0; bool ok = true;
-            int ss = 0; uint32_t sphase = 0;
-            long issued = 0;
-            const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
-            const bool use_a = p.hint_a != 0, use_b = p.hint_b != 0;
-            auto load_a = [&](uint32_t dst, uint32_t bar, int c0, int c1) {
-                if (use_a) tma_load_2d_hint(dst, &tmA, bar, c0, c1, pol_a); else tma_load_2d(dst, &tmA, bar, c0, c1);
-            };
-            auto load_b = [&](uint32_t dst, uint32_t bar, int c0, int c1) {
-                if (use_b) tma_load_2d_hint(dst, &tmB, bar, c0, c1, pol_b); else tma_load_2d(dst, &tmB, bar, c0, c1);
-            };
-            // The loads of one k-block of one tile into a stage.
-            auto issue = [&](int mt, int nt, int kb, uint32_t sa, uint32_t sb, uint32_t bar) {
-                if (A_MN && p.a_3d) {
-                    const int c1 = p.a_k0 + kb * BK, c2 = (p.a_mn0 + mt * BM) >> 6;
-                    if (use_a) tma_load_3d_hint(sa, &tmA, bar, 0, c1, c2, pol_a); else tma_load_3d(sa, &tmA, bar, 0, c1, c2);
-                } else if (A_MN) {
-#pragma unroll
-                    for (int j = 0; j < BM / 64; ++j)
-                        load_a(sa + j * (BK * 128), bar, p.a_mn0 + mt * BM + 64 * j, p.a_k0 + kb * BK);
-                } else {
-                    load_a(sa, bar, p.a_k0 + kb * BK, p.a_mn0 + mt * BM);
-                }
-                if (B_MN && p.b_3d) {
-                    const int c1 = p.b_k0 + kb * BK, c2 = (p.b_mn0 + nt * BN) >> 6;
-                    if (use_b) tma_load_3d_hint(sb, &tmB, bar, 0, c1, c2, pol_b); else tma_load_3d(sb, &tmB, bar, 0, c1, c2);
-                } else if (B_MN) {
-#pragma unroll
-                    for (int j = 0; j < BN / 64; ++j)
-                        load_b(sb + j * (BK * 128), bar, p.b_mn0 + nt * BN + 64 * j, p.b_k0 + kb * BK);
-                } else {
-                    load_b(sb, bar, p.b_k0 + kb * BK, p.b_mn0 + nt * BN);
-                }
-            };
-            while (ok) {
-                if (!mbar_wait(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; break; }
-                int tile = atomicAdd(p.tile_counter, 1);
-                if (tile >= total_tiles) tile = -1;
-                sched_slot[ss] = tile;
-                mbar_arrive(sfull_bar(ss));                              // release: the slot is visible to waiters
-                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
-                if (tile < 0) break;
-                int mt, nt;
-                decode_tile(p, tile, mt, nt);
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
-                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-                    issue(mt, nt, kb, sa, sa + Cfg::A_BYTES, full_bar(stage));
-                    ++issued;
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!ok || *abort_flag) {
-                // Give-up path: let this CTA's copies in flight land before shared memory is released.
-                const long back = issued < STAGES ? issued : STAGES;
-                int s = stage; uint32_t ph = phase;
-                for (long i = 0; i < back; ++i) {
-                    if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
-                    unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0; bool ok = true;
-            int ss = 0; uint32_t sphase = 0;
-            for (int it = 0; ok; ++it) {
-                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
-                const int tile = sched_slot[ss];
-                mbar_arrive(sempty_bar(ss));
-                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
-                if (tile < 0) break;
-                int mt, nt;
-                decode_tile(p, tile, mt, nt);
-                const uint32_t idesc = make_idesc(tile_n(nt), A_MN, B_MN);
-                const int ab = it & 1;
-                const uint32_t aphase = (it >> 1) & 1u;
-                if (!mbar_wait(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-                    const uint32_t sb = sa + Cfg::A_BYTES;
-                    const uint64_t adesc = A_MN ? make_smem_desc(sa, BK * 128, 1024) : make_smem_desc(sa, 16, 1024);
-                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, BK * 128, 1024) : make_smem_desc(sb, 16, 1024);
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // K-major: 16 elements = 32 B along the swizzled row; MN-major: 16 K-rows = 2048 B
-                        const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        umma_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
-                    umma_commit(empty_bar(stage));                      // frees the stage once these MMAs retire
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-                if (ok) umma_commit(tfull_bar(ab));
-            }
-            if (!ok || *abort_flag) {
-                umma_commit(drain_bar);                                 // wait for MMAs still in flight
-                unsigned long long t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
-            }
-        }
-    } else {
-        // ---------------------------------------------------------------- epilogue warps
-        const int quad = warp & 3;                                     // TMEM lane quadrant this warp may read
-        const int row = quad * 32 + lane;
-        int ss = 0; uint32_t sphase = 0;
-        bool ok = true;
-        for (int it = 0; ok; ++it) {
-            int tile = -2;
-            if (lane == 0) {
-                if (mbar_wait(sfull_bar(ss), sphase, abort_flag)) {
-                    tile = sched_slot[ss];
-                    mbar_arrive(sempty_bar(ss));
-                }
-            }
-            tile = __shfl_sync(0xffffffffu, tile, 0);
-            if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
-            if (tile < 0) break;                                        // -1: no tiles left, -2: gave up
-            int mt, nt;
-            decode_tile(p, tile, mt, nt);
-            const int ab = it & 1;
-            const uint32_t aphase = (it >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
-            if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
-            else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh(p, mt, nt * BN, row, tmem_row, tile_n(nt));
-            else epilogue_dw(p, mt, nt * BN, row, tmem_row, tile_n(nt));
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(ab));
-        }
-        if (EPI == EPI_RESID && lane == 0) bulk_wait_all();             // staged stores have landed
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, VPCE_DEV_WAIT_EXPIRED);
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
-    }
-}
-
-// ------------------------------------------------------------------------------------ the CTA-pair GEMM kernel
-// Two CTAs of a cluster (one TPC) work on one 256 x BN tile with tcgen05.mma.cta_group::2: each
-// CTA loads its own 128 rows of A and HALF of the B tile (BN/2 rows), the leader CTA (cluster rank
-// 0) issues the MMAs, which read both CTAs' shared memory and write both CTAs' tensor memory, and
-// each CTA drains its own 128 accumulator rows.  Per CTA and k-block this moves 16 KB + BN*64 B
-// from L2 instead of 16 KB + BN*128 B: a third less L2->SM traffic at BN = 256.
-// Signalling: TMA byte counts of both CTAs are credited to the leader's "full" barrier
-// (.cta_group::2 loads, no multicast); tcgen05.commit with a CTA mask releases the stage in both
-// CTAs and publishes the accumulator to both epilogues; epilogue warps of both CTAs arrive on the
-// leader's "accumulator free" barrier.  Tiles are assigned round-robin to the pairs.
-template <int BN> struct PairCfg {
-    static constexpr int A_BYTES = BM * BK * 2;
-    static constexpr int B_BYTES = (BN / 2) * BK * 2;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
-    static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
-};
-template <int BN, int EPI> constexpr int pair_smem_total() {
-    return PairCfg<BN>::SMEM_TOTAL + (EPI == 1 ? G_STAGING_BYTES : 0);
-}
-
-template <int BN, bool A_MN, bool B_MN, int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-    using Cfg = PairCfg<BN>;
-    constexpr int STAGES = Cfg::STAGES;
-    constexpr uint32_t TMEM_COLS = 512u;
-    constexpr uint32_t ACC_STRIDE = 256u;
-    static_assert(BN == 256, "pair tiles are 256 x 256");
-
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t bars = base + STAGES * Cfg::STAGE_BYTES;
-    auto full_bar = [&](int s) { return bars + 8u * s; };                    // used in the leader only
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
-    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };   // used in the leader only
-    const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
-    auto sfull_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + s); };
-    auto sempty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 5 + SCHED_DEPTH + s); };   // used in the leader only
-    constexpr int NUM_BARS = 2 * STAGES + 5 + 2 * SCHED_DEPTH;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + STAGES * Cfg::STAGE_BYTES + 8 * NUM_BARS);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* sched_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [SCHED_DEPTH] list positions
-    const uint32_t sched_slot_addr = bars + 8u * NUM_BARS + 8u;
-    const uint32_t g_staging = base + STAGES * Cfg::STAGE_BYTES + 1024;
-
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();
-    const bool leader = rank == 0;
-    const int pm_tiles = (p.m_tiles + 1) >> 1;                               // 256-row tiles
-
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
-        mbar_init(drain_bar, 1);
-        // a slot is free again when the leader's MMA lane + 4 epilogue warps and the peer's producer + 4 epilogue
-        // warps have read it: 10 arrivals on the leader's barrier
-        for (int s = 0; s < SCHED_DEPTH; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 10); }
-        fence_barrier_init();
-        fence_proxy_async();
-        prefetch_tensormap(&tmA);
-        prefetch_tensormap(&tmB);
-    }
-    if (warp == 1) {
-        tmem2_alloc(smem_u32(tmem_slot), TMEM_COLS);
-        tmem2_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                                      // the peer's barriers exist before any remote signal
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    // MMA width of n-tile nt.  Each CTA supplies N/2 columns of B: N/2 must be a multiple of 16, and
-    // of 64 (one swizzled chunk) when B is MN-major.
-    auto tile_n = [&](int nt) {
-        const int left = p.cols_valid - nt * BN;
-        constexpr int R = B_MN ? 128 : 32;
-        return left >= BN ? BN : ((left + R - 1) / R * R);
-    };
-    // The work list, longest items first, handed out dynamically (greedy list scheduling):
-    //   [0, n_whole)                  whole 256 x 256 tiles, n-fastest inside raster groups over the full-width n-tiles;
-    //   [n_whole, n_whole + 2*n_cut)  the last n_cut full-width tiles as two 128-column halves each (gradient GEMMs
-    //                                 only, and only when the host's estimate says the last round ends sooner that way);
-    //   the rest                      the narrower last n-tile of every row, when the width is not a multiple of 256.
-    constexpr bool kSplit = (EPI == EPI_DH || EPI == EPI_DW);
-    const int n_wide = p.cols_valid / BN;                                    // full-width n-tiles per row
-    const int n_wide_tiles = pm_tiles * n_wide;
-    const int n_cut = kSplit ? min(p.n_cut, n_wide_tiles) : 0;              // chosen by the host (pick_n_cut)
-    const int n_whole = n_wide_tiles - n_cut;
-    const int n_tail = (p.n_tiles > n_wide) ? pm_tiles : 0;
-    const int list_len = n_whole + 2 * n_cut + n_tail;
-    auto decode_wide = [&](int tile, int& pmt, int& nt) {                    // raster order over the full-width n-tiles
-        const int gn = min(p.group_n, max(n_wide, 1));
-        const int per_group = gn * pm_tiles;
-        const int g = tile / per_group;
-        const int r = tile - g * per_group;
-        const int n0 = g * gn;
-        const int gw = min(gn, n_wide - n0);
-        pmt = r / gw;
-        nt = n0 + (r - pmt * gw);
-    };
-    auto get_tile = [&](int t, int& pmt, int& nt, int& ncol0, int& width) {
-        if (t < n_whole) {
-            decode_wide(t, pmt, nt);
-            ncol0 = nt * BN; width = BN;
-        } else if (t < n_whole + 2 * n_cut) {
-            const int v = t - n_whole;
-            decode_wide(n_whole + (v >> 1), pmt, nt);
-            ncol0 = nt * BN + (v & 1) * (BN / 2); width = BN / 2;
-        } else {
-            pmt = t - (n_whole + 2 * n_cut);
-            nt = n_wide;
-            ncol0 = nt * BN; width = tile_n(nt);
-        }
-    };
-    // Scheduler ring: the leader's producer lane takes list positions from the launch's counter and writes them
-    // into the same slot of both CTAs; every reader acknowledges on the leader's "slot free" barrier.
-    auto sched_ack = [&](int ss) { mbar_arrive_cluster(mapa_shared(sempty_bar(ss), 0)); };
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- scheduler (leader) + TMA producer (both CTAs)
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0; bool ok = true;
-            int ss = 0; uint32_t sphase = 0;
-            long issued = 0;
-            const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
-            while (ok) {
-                int tile;
-                if (leader) {
-                    if (!mbar_wait_cluster(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; break; }
-                    tile = atomicAdd(p.tile_counter, 1);
-                    if (tile >= list_len) tile = -1;
-                    sched_slot[ss] = tile;
-                    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(sched_slot_addr + 4u * ss, 1)), "r"(tile) : "memory");
-                    mbar_arrive(sfull_bar(ss));
-                    mbar_arrive_cluster(mapa_shared(sfull_bar(ss), 1));      // release.cluster: the peer sees its slot
-                } else {
-                    if (!mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
-                    tile = sched_slot[ss];
-                    sched_ack(ss);
-                }
-                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
-                if (tile < 0) break;
-                int pmt, nt, ncol0, width;
-                get_tile(tile, pmt, nt, ncol0, width);
-                const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
-                const int bn0 = ncol0 + static_cast<int>(rank) * (width / 2);   // this CTA's half of the B tile
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
-                    const uint32_t bar = mapa_shared(full_bar(stage), 0);    // the leader's barrier
-                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-                    const uint32_t sb = sa + Cfg::A_BYTES;
-                    if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BK, (p.a_mn0 + mt * BM) >> 6, pol_a);
-                    else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BK, p.a_mn0 + mt * BM, pol_a);
-                    if (B_MN) tma2_load_3d(sb, &tmB, bar, 0, p.b_k0 + kb * BK, (p.b_mn0 + bn0) >> 6, pol_b);
-                    else tma2_load_2d(sb, &tmB, bar, p.b_k0 + kb * BK, p.b_mn0 + bn0, pol_b);
-                    ++issued;
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if ((!ok || *abort_flag) && leader) {
-                // Give-up path (the leader's barriers count both CTAs' bytes): let copies in flight land.
-                const long back = issued < STAGES ? issued : STAGES;
-                int s = stage; uint32_t ph = phase;
-                for (long i = 0; i < back; ++i) {
-                    if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
-                    unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer (leader CTA only)
-        if (lane == 0 && leader) {
-            int stage = 0; uint32_t phase = 0; bool ok = true;
-            int ss = 0; uint32_t sphase = 0;
-            for (int it = 0; ok; ++it) {
-                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
-                const int tile = sched_slot[ss];
-                sched_ack(ss);
-                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
-                if (tile < 0) break;
-                int pmt, nt, ncol0, width;
-                get_tile(tile, pmt, nt, ncol0, width);
-                const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM);
-                const int ab = it & 1;
-                const uint32_t aphase = (it >> 1) & 1u;
-                if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-                    const uint32_t sb = sa + Cfg::A_BYTES;
-                    const uint64_t adesc = A_MN ? make_smem_desc(sa, BK * 128, 1024) : make_smem_desc(sa, 16, 1024);
-                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, BK * 128, 1024) : make_smem_desc(sb, 16, 1024);
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        umma2_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
-                    umma2_commit_both(empty_bar(stage));                     // frees the stage in both CTAs
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-                if (ok) umma2_commit_both(tfull_bar(ab));                    // accumulator ready in both CTAs
-            }
-            if (!ok || *abort_flag) {
-                umma2_commit_local(drain_bar);
-                unsigned long long t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < WAIT_LIMIT_NS) {}
-            }
-        }
-    } else {
-        // ---------------------------------------------------------------- epilogue warps (both CTAs)
-        const int quad = warp & 3;
-        const int row = quad * 32 + lane;
-        int ss = 0; uint32_t sphase = 0;
-        bool ok = true;
-        for (int it = 0; ok; ++it) {
-            int tile = -2;
-            if (lane == 0) {
-                if (mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) {
-                    tile = sched_slot[ss];
-                    sched_ack(ss);
-                }
-            }
-            tile = __shfl_sync(0xffffffffu, tile, 0);
-            if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
-            if (tile < 0) break;                                             // -1: list exhausted, -2: gave up
-            int pmt, nt, ncol0, width;
-            get_tile(tile, pmt, nt, ncol0, width);
-            const int mt = 2 * pmt + static_cast<int>(rank);
-            const int ab = it & 1;
-            const uint32_t aphase = (it >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
-            if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
-            else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh(p, mt, ncol0, row, tmem_row, width);
-            else epilogue_dw(p, mt, ncol0, row, tmem_row, width);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
-        }
-        if (EPI == EPI_RESID && lane == 0) bulk_wait_all();
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                          // no CTA leaves while its pair may still signal it or read its memory
-    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, VPCE_DEV_WAIT_EXPIRED);
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        tmem2_dealloc(tmem_base, TMEM_COLS);
-    }
-}
-
-// ------------------------------------------------------------------------------------ small kernels
-// Folds the per-tile partial states of one strip into the running per-token state (Eq. 2
-// applied to two states: m = max(m1, m2), z = z1 e^{m1-m} + z2 e^{m2-m}), in tile order so the
-// result does not depend on which CTA produced which tile.  On the last step it also emits
-// lse = m + log z and loss = lse - y_t (Algorithm 3, output line).
-__global__ void vpce_merge_kernel(const float* __restrict__ pm, const float* __restrict__ pz, int part_ld, int n_tiles,
-                                  float* __restrict__ sm, float* __restrict__ sz, const float* __restrict__ ylab,
-                                  int rows, int first, int last, const int32_t* __restrict__ labels, int ignore_index,
-                                  int V, float* __restrict__ lse, float* __restrict__ loss, int* status) {
-    const int n = blockIdx.x * blockDim.x + threadIdx.x;
-    if (n >= rows) return;
-    float m = first ? NEG_INF : sm[n];
-    float z = first ? 0.f : sz[n];
-    for (int t = 0; t < n_tiles; ++t) {
-        const float m2 = pm[static_cast<size_t>(t) * part_ld + n];
-        const float z2 = pz[static_cast<size_t>(t) * part_ld + n];
-        const float mn = fmaxf(m, m2);
-        z = z * ex2f((m - mn) * LOG2E) + z2 * ex2f((m2 - mn) * LOG2E);   // m = -inf contributes 0
-        m = mn;
-    }
-    if (!last) { sm[n] = m; sz[n] = z; return; }
-    const float l = m + logf(z);
-    lse[n] = l;
-    const int t = labels[n];
-    float out = 0.f;
-    if (t != ignore_index) {
-        if (static_cast<unsigned>(t) < static_cast<unsigned>(V)) out = l - ylab[n];
-        else atomicOr(status, VPCE_DEV_LABEL_OUT_OF_RANGE);
-    }
-    loss[n] = out;
-}
-
-// One block: counts valid labels (fixed order) and stores 1 / n_valid (0 when there is none).
-__global__ void vpce_count_valid_kernel(const int32_t* __restrict__ labels, long T, int V, int ignore_index,
-                                        float* inv_n_valid, int* n_valid_out, int* status) {
-    __shared__ int part[1024];
-    int c = 0, bad = 0;
-    for (long i = threadIdx.x; i < T; i += blockDim.x) {
-        const int t = labels[i];
-        if (t != ignore_index) {
-            if (static_cast<unsigned>(t) < static_cast<unsigned>(V)) ++c; else bad = 1;
-        }
-    }
-    if (bad && status) atomicOr(status, VPCE_DEV_LABEL_OUT_OF_RANGE);
-    part[threadIdx.x] = c;
-    __syncthreads();
-    for (int s = blockDim.x / 2; s > 0; s >>= 1) {
-        if (threadIdx.x < s) part[threadIdx.x] += part[threadIdx.x + s];
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        if (inv_n_valid) *inv_n_valid = part[0] > 0 ? 1.0f / static_cast<float>(part[0]) : 0.f;
-        if (n_valid_out) *n_valid_out = part[0];
-    }
-}
-
-// One block: masked mean of the per-token loss, double accumulation in a fixed order.
-__global__ void vpce_mean_loss_kernel(const float* __restrict__ loss, const int32_t* __restrict__ labels, long T, int V,
-                                      int ignore_index, float* mean_out, int* n_valid_out) {
-    __shared__ double sums[1024];
-    __shared__ int cnts[1024];
-    double s = 0.0; int c = 0;
-    for (long i = threadIdx.x; i < T; i += blockDim.x) {
-        const int t = labels[i];
-        if (t != ignore_index && static_cast<unsigned>(t) < static_cast<unsigned>(V)) { s += loss[i]; ++c; }
-    }
-    sums[threadIdx.x] = s; cnts[threadIdx.x] = c;
-    __syncthreads();
-    for (int k = blockDim.x / 2; k > 0; k >>= 1) {
-        if (threadIdx.x < k) { sums[threadIdx.x] += sums[threadIdx.x + k]; cnts[threadIdx.x] += cnts[threadIdx.x + k]; }
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        *mean_out = cnts[0] > 0 ? static_cast<float>(sums[0] / cnts[0]) : 0.f;
-        *n_valid_out = cnts[0];
-    }
-}
-
-__global__ void vpce_clear_status_kernel(int* status) { if (threadIdx.x < 8) status[threadIdx.x] = 0; }
+using namespace vpce;
 
 // ------------------------------------------------------------------------------------ host side
 std::atomic<long long> g_launches{0};
