@@ -561,41 +561,39 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         constexpr int R = B_MN ? 128 : 32;
         return left >= BN ? BN : ((left + R - 1) / R * R);
     };
-    // The work list, longest items first, handed out dynamically (greedy list scheduling):
-    //   [0, n_whole)                  whole 256 x 256 tiles, n-fastest inside raster groups over the full-width n-tiles;
-    //   [n_whole, n_whole + 2*n_cut)  the last n_cut full-width tiles as two 128-column halves each (gradient GEMMs
-    //                                 only, and only when the host's estimate says the last round ends sooner that way);
-    //   the rest                      the narrower last n-tile of every row, when the width is not a multiple of 256.
+    // The work list, handed out dynamically (greedy list scheduling):
+    //   [0, n_whole)                  256-row x BN tiles in raster order: n-fastest over ALL n-tiles of a row inside
+    //                                 raster groups, so the narrower last n-tile of a row runs next to the row's other
+    //                                 tiles and shares their A rows through L2 (placing those tiles at the end of the
+    //                                 list re-read the whole A operand from DRAM);
+    //   [n_whole, n_whole + 2*n_cut)  the last n_cut tiles as two 128-column halves each (gradient GEMMs only, and only
+    //                                 when the host's estimate says the last round ends sooner that way).
     constexpr bool kSplit = (EPI == EPI_DH || EPI == EPI_DW);
-    const int n_wide = p.cols_valid / BN;                                    // full-width n-tiles per row
-    const int n_wide_tiles = pm_tiles * n_wide;
-    const int n_cut = kSplit ? min(p.n_cut, n_wide_tiles) : 0;              // chosen by the host (pick_n_cut)
-    const int n_whole = n_wide_tiles - n_cut;
-    const int n_tail = (p.n_tiles > n_wide) ? pm_tiles : 0;
-    const int list_len = n_whole + 2 * n_cut + n_tail;
-    auto decode_wide = [&](int tile, int& pmt, int& nt) {                    // raster order over the full-width n-tiles
-        const int gn = min(p.group_n, max(n_wide, 1));
-        const int per_group = gn * pm_tiles;
+    const int total_tiles = pm_tiles * p.n_tiles;
+    const int n_cut = kSplit ? min(p.n_cut, total_tiles) : 0;
+    const int n_whole = total_tiles - n_cut;
+    const int list_len = n_whole + 2 * n_cut;
+    auto decode_raster = [&](int tile, int& pmt, int& nt) {
+        const int per_group = p.group_n * pm_tiles;
         const int g = tile / per_group;
         const int r = tile - g * per_group;
-        const int n0 = g * gn;
-        const int gw = min(gn, n_wide - n0);
+        const int n0 = g * p.group_n;
+        const int gw = min(p.group_n, p.n_tiles - n0);
         pmt = r / gw;
         nt = n0 + (r - pmt * gw);
     };
+    // Entry t of the list: 256-row tile pmt, columns [ncol0, ncol0 + width) of n-tile nt; width == 0 means "nothing".
     auto get_tile = [&](int t, int& pmt, int& nt, int& ncol0, int& width) {
         if (t < n_whole) {
-            decode_wide(t, pmt, nt);
-            ncol0 = nt * BN; width = BN;
-        } else if (t < n_whole + 2 * n_cut) {
-            const int v = t - n_whole;
-            decode_wide(n_whole + (v >> 1), pmt, nt);
-            ncol0 = nt * BN + (v & 1) * (BN / 2); width = BN / 2;
-        } else {
-            pmt = t - (n_whole + 2 * n_cut);
-            nt = n_wide;
+            decode_raster(t, pmt, nt);
             ncol0 = nt * BN; width = tile_n(nt);
+            return;
         }
+        const int v = t - n_whole;
+        decode_raster(n_whole + (v >> 1), pmt, nt);
+        const int w = tile_n(nt);
+        if (w <= BN / 2) { ncol0 = nt * BN; width = (v & 1) ? 0 : w; }
+        else { ncol0 = nt * BN + (v & 1) * (BN / 2); width = (v & 1) ? w - BN / 2 : BN / 2; }
     };
     // Scheduler ring: the leader's producer lane takes list positions from the launch's counter and writes them
     // into the same slot of both CTAs; every reader acknowledges on the leader's "slot free" barrier.
@@ -627,6 +625,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (tile < 0) break;
                 int pmt, nt, ncol0, width;
                 get_tile(tile, pmt, nt, ncol0, width);
+                if (width == 0) continue;
                 const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
                 const int bn0 = ncol0 + static_cast<int>(rank) * (width / 2);   // this CTA's half of the B tile
                 for (int kb = 0; kb < p.num_kb; ++kb) {
@@ -659,7 +658,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         if (lane == 0 && leader) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             int ss = 0; uint32_t sphase = 0;
-            for (int it = 0; ok; ++it) {
+            for (int it = 0; ok;) {
                 if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
                 const int tile = sched_slot[ss];
                 sched_ack(ss);
@@ -667,6 +666,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (tile < 0) break;
                 int pmt, nt, ncol0, width;
                 get_tile(tile, pmt, nt, ncol0, width);
+                if (width == 0) continue;
                 const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
@@ -690,6 +690,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (ok) umma2_commit_both(tfull_bar(ab));                    // accumulator ready in both CTAs
+                ++it;
             }
             if (!ok || *abort_flag) {
                 umma2_commit_local(drain_bar);
@@ -703,7 +704,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         const int row = quad * 32 + lane;
         int ss = 0; uint32_t sphase = 0;
         bool ok = true;
-        for (int it = 0; ok; ++it) {
+        for (int it = 0; ok;) {
             int tile = -2;
             if (lane == 0) {
                 if (mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) {
@@ -716,6 +717,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (tile < 0) break;                                             // -1: list exhausted, -2: gave up
             int pmt, nt, ncol0, width;
             get_tile(tile, pmt, nt, ncol0, width);
+            if (width == 0) continue;
             const int mt = 2 * pmt + static_cast<int>(rank);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
@@ -729,6 +731,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
+            ++it;
         }
         if (EPI == EPI_RESID && lane == 0) bulk_wait_all();
     }
