@@ -209,8 +209,8 @@ __device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nco
             if (col0 + 8 * q >= p.cols_valid) break;                   // d is a multiple of 8
             float* x = v + 8 * q;
             if (!p.first) {
-                const float4 a0 = *reinterpret_cast<const float4*>(arow + 8 * q);
-                const float4 a1 = *reinterpret_cast<const float4*>(arow + 8 * q + 4);
+                const float4 a0 = __ldcs(reinterpret_cast<const float4*>(arow + 8 * q));      // streamed: read once
+                const float4 a1 = __ldcs(reinterpret_cast<const float4*>(arow + 8 * q + 4));
                 x[0] += a0.x; x[1] += a0.y; x[2] += a0.z; x[3] += a0.w;
                 x[4] += a1.x; x[5] += a1.y; x[6] += a1.z; x[7] += a1.w;
             }
@@ -218,10 +218,10 @@ __device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int nco
                 uint4 o;
                 o.x = pack_bf16x2(x[0], x[1]); o.y = pack_bf16x2(x[2], x[3]);
                 o.z = pack_bf16x2(x[4], x[5]); o.w = pack_bf16x2(x[6], x[7]);
-                *reinterpret_cast<uint4*>(orow + 8 * q) = o;
+                __stcs(reinterpret_cast<uint4*>(orow + 8 * q), o);
             } else {
-                *reinterpret_cast<float4*>(arow + 8 * q) = make_float4(x[0], x[1], x[2], x[3]);
-                *reinterpret_cast<float4*>(arow + 8 * q + 4) = make_float4(x[4], x[5], x[6], x[7]);
+                __stcs(reinterpret_cast<float4*>(arow + 8 * q), make_float4(x[0], x[1], x[2], x[3]));
+                __stcs(reinterpret_cast<float4*>(arow + 8 * q + 4), make_float4(x[4], x[5], x[6], x[7]));
             }
         }
         }
@@ -245,10 +245,10 @@ __device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nco
             if (col0 + 4 * q >= p.cols_valid) break;
             float4 x = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
             if (p.accumulate) {
-                const float4 a = *reinterpret_cast<const float4*>(orow + 4 * q);
+                const float4 a = __ldcs(reinterpret_cast<const float4*>(orow + 4 * q));
                 x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
             }
-            *reinterpret_cast<float4*>(orow + 4 * q) = x;
+            __stcs(reinterpret_cast<float4*>(orow + 4 * q), x);                     // streamed: not re-read by this launch
         }
         }
     }
