@@ -260,7 +260,7 @@ __device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int nco
 // shared-memory ring guarded by mbarriers, so a CTA that finishes early simply takes more tiles.
 // The last n-tile of a row may be narrower than BN (its MMA uses N = valid columns rounded up
 // to 16), so an output width that is not a multiple of BN costs no padded tensor-core work.
-constexpr int SCHED_DEPTH = 4;
+constexpr int SCHED_DEPTH = 8;
 
 template <int BN, bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -606,22 +606,34 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int ss = 0; uint32_t sphase = 0;
             long issued = 0;
             const uint64_t pol_a = make_policy(p.hint_a), pol_b = make_policy(p.hint_b);
+            // Leader: take the next list position and publish it to both CTAs.  It runs one entry ahead of the
+            // loads (the atomic's latency hides behind the copies of the current tile).
+            bool exhausted = false;
+            auto publish = [&]() -> int {
+                if (exhausted) return -1;
+                if (!mbar_wait_cluster(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; return -1; }
+                int t = atomicAdd(p.tile_counter, 1);
+                if (t >= list_len) { t = -1; exhausted = true; }
+                sched_slot[ss] = t;
+                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(sched_slot_addr + 4u * ss, 1)), "r"(t) : "memory");
+                mbar_arrive(sfull_bar(ss));
+                mbar_arrive_cluster(mapa_shared(sfull_bar(ss), 1));          // release.cluster: the peer sees its slot
+                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
+                return t;
+            };
+            int ahead = leader ? publish() : 0;
             while (ok) {
                 int tile;
                 if (leader) {
-                    if (!mbar_wait_cluster(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; break; }
-                    tile = atomicAdd(p.tile_counter, 1);
-                    if (tile >= list_len) tile = -1;
-                    sched_slot[ss] = tile;
-                    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(mapa_shared(sched_slot_addr + 4u * ss, 1)), "r"(tile) : "memory");
-                    mbar_arrive(sfull_bar(ss));
-                    mbar_arrive_cluster(mapa_shared(sfull_bar(ss), 1));      // release.cluster: the peer sees its slot
+                    tile = ahead;
+                    if (tile >= 0) ahead = publish();
+                    if (!ok) break;
                 } else {
                     if (!mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
                     tile = sched_slot[ss];
                     sched_ack(ss);
+                    if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
                 }
-                if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
                 if (tile < 0) break;
                 int pmt, nt, ncol0, width;
                 get_tile(tile, pmt, nt, ncol0, width);
