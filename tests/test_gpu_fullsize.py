@@ -18,7 +18,7 @@ from bench import BENCH_T_CHUNK
 from oracle import vpce_oracle as orc
 from synth_inputs import (IGNORE_INDEX, WORKLOADS, bf16_bits_to_f64, make_hidden, make_weights,
                           stream_labels)
-from vpce_testlib import TOL_GRAD, TOL_TOKEN, GpuRun, relF
+from vpce_testlib import TOL_GRAD, TOL_TOKEN, DeviceRun, relF
 
 pytestmark = pytest.mark.gpu
 
@@ -46,7 +46,7 @@ def check_call(w, call, W_bits, W64, labels_stream, n_valid_total, T_chunk, W_de
     H_bits = make_hidden(w, call)
     labels = labels_stream[call * w.T:(call + 1) * w.T]
     base = call * (-(-w.T // T_chunk))
-    run = GpuRun(H_bits, W_bits, labels, w.block_v, T_chunk, base, W_dev=W_dev)
+    run = DeviceRun(H_bits, W_bits, labels, w.block_v, T_chunk, base, W_dev=W_dev)
     run.forward()
     assert run.fwd_status == 0
     # ---- default (masked-mean over the stream) upstream gradient: lse, loss, dH on sampled tokens

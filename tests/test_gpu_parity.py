@@ -9,7 +9,7 @@ import paper_2609_14306_b200 as vp
 from oracle import vpce_oracle as orc
 from synth_inputs import (IGNORE_INDEX, WORKLOADS, bf16_bits_to_f64, custom_workload, make_batch,
                           make_dloss)
-from vpce_testlib import (TOL_GRAD, TOL_TOKEN, GpuRun, check_against_oracle, relF)
+from vpce_testlib import (TOL_GRAD, TOL_TOKEN, DeviceRun, check_against_oracle, relF)
 
 pytestmark = pytest.mark.gpu
 
@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 def full_check(w, dloss=None, base=0, tag=None):
     b = make_batch(w)
     H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
-    run = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk, base).forward().backward(dloss)
+    run = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk, base).forward().backward(dloss)
     assert run.fwd_status == 0 and run.bwd_status == 0
     ref = orc.forward_backward(H64, W64, b.labels, dloss, IGNORE_INDEX)
     dl64 = orc.default_dloss(b.labels, IGNORE_INDEX) if dloss is None else dloss.astype(np.float64)
@@ -65,7 +65,7 @@ def test_all_tokens_ignored():
     w = custom_workload("allign", T=256, d=128, V=1024, block_v=512, T_chunk=128, w_std=0.1, seed=5)
     b = make_batch(w)
     lab = np.full(w.T, IGNORE_INDEX, dtype=np.int32)
-    run = GpuRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward()
+    run = DeviceRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward()
     lse_ref, _ = orc.dense_forward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), lab)
     assert np.abs(run.np_lse() - lse_ref).max() <= TOL_TOKEN
     assert not run.np_loss().any() and not run.np_dH().any() and not run.np_dW().any()
@@ -75,7 +75,7 @@ def test_all_tokens_ignored():
 def test_zero_weight_gives_log_V():
     w = custom_workload("w0", T=256, d=128, V=1536, block_v=512, T_chunk=128, seed=6, ignore_frac=0.1)
     b = make_batch(w)
-    run = GpuRun(b.H_bits, np.zeros_like(b.W_bits), b.labels, w.block_v, w.T_chunk).forward().backward()
+    run = DeviceRun(b.H_bits, np.zeros_like(b.W_bits), b.labels, w.block_v, w.T_chunk).forward().backward()
     valid = b.labels != IGNORE_INDEX
     assert np.abs(run.np_lse() - np.log(w.V)).max() < 1e-5
     assert np.abs(run.np_loss()[valid] - np.log(w.V)).max() < 1e-5
@@ -88,7 +88,7 @@ def test_label_out_of_range_sets_status_and_is_ignored():
     lab = b.labels.copy()
     lab[3] = w.V + 5
     lab[200] = -7
-    run = GpuRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward()
+    run = DeviceRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward()
     assert run.fwd_status & 1 and run.bwd_status & 1
     lab_ok = lab.copy()
     lab_ok[[3, 200]] = IGNORE_INDEX
@@ -96,7 +96,7 @@ def test_label_out_of_range_sets_status_and_is_ignored():
     assert np.abs(run.np_loss() - ref["loss"]).max() <= TOL_TOKEN
     assert relF(run.np_dW(), ref["dW"]) <= TOL_GRAD and relF(run.np_dH(), ref["dH"]) <= TOL_GRAD
     # a later clean call clears the flag
-    run2 = GpuRun(b.H_bits, b.W_bits, lab_ok, w.block_v, w.T_chunk).forward()
+    run2 = DeviceRun(b.H_bits, b.W_bits, lab_ok, w.block_v, w.T_chunk).forward()
     assert run2.fwd_status == 0
 
 
@@ -108,7 +108,7 @@ def test_invariance_to_block_chunk_and_rotation():
     ref = orc.forward_backward(H64, W64, b.labels)
     outs = []
     for block_v, T_chunk, base in [(512, 128, 0), (1024, 256, 5), (256, 512, 1), (3072, 128, 2), (4096, 384, 0)]:
-        r = GpuRun(b.H_bits, b.W_bits, b.labels, block_v, T_chunk, base).forward().backward()
+        r = DeviceRun(b.H_bits, b.W_bits, b.labels, block_v, T_chunk, base).forward().backward()
         assert np.abs(r.np_lse() - ref["lse"]).max() <= TOL_TOKEN
         assert relF(r.np_dH(), ref["dH"]) <= TOL_GRAD and relF(r.np_dW(), ref["dW"]) <= TOL_GRAD
         outs.append(r.np_lse())
@@ -120,8 +120,8 @@ def test_invariance_to_block_chunk_and_rotation():
 def test_run_to_run_bitwise_determinism():
     w = WORKLOADS["tiny"]
     b = make_batch(w)
-    a = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
-    c = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
+    a = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
+    c = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
     assert torch.equal(a.lse, c.lse) and torch.equal(a.loss, c.loss)
     assert torch.equal(a.dH.view(torch.int16), c.dH.view(torch.int16)) and torch.equal(a.dW, c.dW)
 
@@ -140,7 +140,7 @@ def test_accumulate_dW_across_calls_matches_one_call():
     parts = []
     for k in range(2):
         sl = slice(k * half, (k + 1) * half)
-        r = GpuRun(b.H_bits[sl], b.W_bits, b.labels[sl], w.block_v, w.T_chunk, chunk_index_base=k * (half // w.T_chunk),
+        r = DeviceRun(b.H_bits[sl], b.W_bits, b.labels[sl], w.block_v, w.T_chunk, chunk_index_base=k * (half // w.T_chunk),
                    W_dev=Wd, dW=dW)
         Wd = r.W
         r.forward().backward(dloss=dl[sl].astype(np.float32), accumulate=True)
@@ -153,7 +153,7 @@ def test_accumulate_dW_across_calls_matches_one_call():
 def test_host_side_argument_checks():
     w = WORKLOADS["tiny"]
     b = make_batch(w)
-    r = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
+    r = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
     small = torch.empty(1024, dtype=torch.uint8, device="cuda")
     with pytest.raises(vp.VpceError) as ei:
         vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, 0, small)
@@ -180,7 +180,7 @@ def test_degenerate_small_shapes(T, d, V, block_v, T_chunk):
                         labels="uniform", ignore_frac=0.0, seed=T * 7 + V)
     b = make_batch(w)
     H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
-    run = GpuRun(b.H_bits, b.W_bits, b.labels, block_v, T_chunk).forward().backward()
+    run = DeviceRun(b.H_bits, b.W_bits, b.labels, block_v, T_chunk).forward().backward()
     assert run.fwd_status == 0 and run.bwd_status == 0
     ref = orc.forward_backward(H64, W64, b.labels)
     assert np.abs(run.np_lse() - ref["lse"]).max() <= TOL_TOKEN
@@ -195,7 +195,7 @@ def test_degenerate_small_shapes(T, d, V, block_v, T_chunk):
 def test_empty_batch_is_a_no_op():
     w = custom_workload("empty", T=128, d=64, V=512, block_v=256, T_chunk=128, seed=3)
     b = make_batch(w)
-    r = GpuRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
+    r = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
     H0 = r.H[:0].contiguous()
     lab0 = r.labels[:0].contiguous()
     out0 = torch.empty(0, dtype=torch.float32, device="cuda")

@@ -21,7 +21,7 @@ def relF(a: np.ndarray, ref: np.ndarray) -> float:
     return num / den if den > 0 else num
 
 
-class GpuRun:
+class DeviceRun:
     """Device buffers and results of one forward(+backward) call."""
 
     def __init__(self, H_bits, W_bits, labels, block_v, T_chunk, chunk_index_base=0, ignore_index=IGNORE_INDEX,
@@ -87,7 +87,7 @@ def softmax_only_residuals(dH, dW, H64, W64, labels, dloss64, ignore_index=IGNOR
     return dH_s, dW_s
 
 
-def check_against_oracle(run: GpuRun, ref: dict, H64, W64, labels, dloss64, tag=""):
+def check_against_oracle(run: DeviceRun, ref: dict, H64, W64, labels, dloss64, tag=""):
     """Asserts the acceptance tolerances and returns the measured errors."""
     e = {}
     e["lse"] = float(np.abs(run.np_lse() - ref["lse"]).max())
