@@ -31,9 +31,15 @@ def load_library() -> ctypes.CDLL:
         return _LIB
     path = library_path()
     if not os.path.exists(path):
-        raise RuntimeError(
-            f"{path} is missing: build it with `python -m paper_2609_14306_b200.build` "
-            "(or __graft_entry__.build()); this package has no CPU fallback")
+        # Not built yet: compile it in-tree now (nvcc, sm_100a).  There is no other implementation to fall
+        # back to, so a failed build is fatal.
+        try:
+            from .build import build_library
+            build_library()
+        except Exception as exc:
+            raise RuntimeError(
+                f"{path} is missing and could not be built ({exc}); build it with "
+                "`python -m paper_2609_14306_b200.build`; this package has no CPU fallback") from exc
     lib = ctypes.CDLL(path)
     i64, i32, vp, sz = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t
     lib.vp_ce_workspace_bytes.restype = sz
