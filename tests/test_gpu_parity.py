@@ -209,3 +209,37 @@ def test_empty_batch_is_a_no_op():
                       w.block_v, IGNORE_INDEX, w.T_chunk, 0, False, r.ws)
     torch.cuda.synchronize()
     assert not dW.any()                                                # overwrite: zero contribution
+
+
+def test_single_cta_kernels_agree_with_pair_kernels():
+    """The library picks CTA-pair kernels by default; VPCE_PAIR=0 forces the one-CTA kernels for every GEMM.
+    Both must meet the tolerances on the same problem (run in a child process: the switch is read per call,
+    but a separate process also proves the fallback path works from a cold start)."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import numpy as np, sys, os
+sys.path.insert(0, os.getcwd()); sys.path.insert(0, os.path.join(os.getcwd(), "tests"))
+from oracle import vpce_oracle as orc
+from synth_inputs import IGNORE_INDEX, bf16_bits_to_f64, custom_workload, make_batch
+from vpce_testlib import DeviceRun, relF
+w = custom_workload("fallback", T=1024, d=2880, V=3000, block_v=1024, T_chunk=512, w_std=0.02, labels="zipf",
+                    ignore_frac=0.05, seed=21)
+b = make_batch(w)
+r = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk, 1).forward().backward()
+ref = orc.forward_backward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), b.labels)
+print(float(np.abs(r.np_lse() - ref["lse"]).max()), float(np.abs(r.np_loss() - ref["loss"]).max()),
+      relF(r.np_dH(), ref["dH"]), relF(r.np_dW(), ref["dW"]), r.fwd_status, r.bwd_status)
+'''
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = {}
+    for mode in ("0", "7"):
+        env = dict(os.environ, VPCE_PAIR=mode)
+        res = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+        assert res.returncode == 0, res.stderr[-2000:]
+        vals = [float(x) for x in res.stdout.strip().split()[-6:]]
+        assert vals[0] <= TOL_TOKEN and vals[1] <= TOL_TOKEN and vals[2] <= TOL_GRAD and vals[3] <= TOL_GRAD, (mode, vals)
+        assert vals[4] == 0 and vals[5] == 0
+        outs[mode] = vals
+    print(outs)
