@@ -231,8 +231,11 @@ int pick_n_cut(int pm_tiles, int n_tiles, int pairs) {
 // Which GEMMs run as CTA pairs (bit 0 strip kernels, bit 1 input-gradient, bit 2 weight-gradient).
 // All of them by default; VPCE_PAIR in the environment overrides it for A/B measurements.
 int pair_mask() {
-    const char* e = getenv("VPCE_PAIR");
-    return e ? atoi(e) : 7;
+    static const int mask = [] {
+        const char* e = getenv("VPCE_PAIR");
+        return e ? atoi(e) : 7;
+    }();
+    return mask;
 }
 
 // Output-column tile for the two gradient GEMMs: 256 unless d is narrower; the last tile of a

@@ -243,3 +243,18 @@ print(float(np.abs(r.np_lse() - ref["lse"]).max()), float(np.abs(r.np_loss() - r
         assert vals[4] == 0 and vals[5] == 0
         outs[mode] = vals
     print(outs)
+
+
+def test_large_logits_stay_finite_and_accurate():
+    # logits of magnitude ~1e2..1e3: the running maximum keeps every exponent argument <= 0
+    w = custom_workload("big", T=256, d=256, V=2048, block_v=512, T_chunk=256, w_std=4.0,
+                        labels="uniform", ignore_frac=0.0, seed=31)
+    b = make_batch(w)
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    run = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk).forward().backward()
+    ref = orc.forward_backward(H64, W64, b.labels)
+    assert np.abs(H64 @ W64.T).max() > 200.0
+    assert np.isfinite(run.np_lse()).all() and np.isfinite(run.np_dW()).all() and np.isfinite(run.np_dH()).all()
+    # fp32 logits of this size carry ~1e-5 relative error, so compare relatively
+    assert np.abs(run.np_lse() - ref["lse"]).max() <= 2e-5 * np.abs(ref["lse"]).max() + TOL_TOKEN
+    assert relF(run.np_dH(), ref["dH"]) <= TOL_GRAD and relF(run.np_dW(), ref["dW"]) <= TOL_GRAD
