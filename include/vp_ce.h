@@ -169,6 +169,26 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
                                  int32_t* device_status_out, void* stream);
 
 /*
+ * FP32-input variants (TF32 tensor cores, fp32 accumulation): the precision of the paper's isolated
+ * Ring-DTP benchmark (Appendix C states FP32; whether its matmuls used TF32 is not stated).  Same
+ * method, semantics, status codes and workspace rules as vp_ce_forward / vp_ce_backward, except:
+ *   H [T, d], W [V, d] are float32; dH [T, d] is float32 (it also serves as the running
+ *   accumulator across shards); the residual strip in the workspace is float32, so
+ *   vp_ce_workspace_bytes_f32 is about twice as large minus the separate accumulator;
+ *   d must be a multiple of 32.  The tensor core reads the upper 19 bits of each input.
+ */
+size_t vp_ce_workspace_bytes_f32(int64_t T_chunk, int64_t d, int64_t block_v);
+vpce_status vp_ce_forward_f32(const float* H, const float* W, const int32_t* labels,
+                              int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                              float* loss, float* lse, int64_t T_chunk, int64_t chunk_index_base,
+                              void* workspace, size_t workspace_bytes, void* stream);
+vpce_status vp_ce_backward_f32(const float* H, const float* W, const int32_t* labels, const float* lse,
+                               const float* dloss, float* dH, float* dW,
+                               int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                               int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Measurement aid (no counterpart in the paper).  While enabled, every tensor-core kernel
  * launch is bracketed by two CUDA events on the launching stream.  vp_ce_profile_collect
  * waits for the recorded events, adds up the elapsed milliseconds and launch counts per kernel

@@ -10,7 +10,10 @@ from .binding import (  # noqa: F401
     vp_ce_backward,
     vp_ce_device_status,
     vp_ce_forward,
+    vp_ce_backward_f32,
+    vp_ce_forward_f32,
     vp_ce_forward_static,
+    vp_ce_workspace_bytes_f32,
     vp_ce_fwd_bwd_host,
     vp_ce_profile_collect,
     vp_ce_profile_enable,

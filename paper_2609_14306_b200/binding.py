@@ -62,6 +62,13 @@ def load_library() -> ctypes.CDLL:
                                        vp, vp, vp, vp, vp, vp, sz, vp]
     lib.vp_ce_forward_static.restype = ctypes.c_int
     lib.vp_ce_forward_static.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, i64, i64, vp, vp]
+    lib.vp_ce_workspace_bytes_f32.restype = sz
+    lib.vp_ce_workspace_bytes_f32.argtypes = [i64, i64, i64]
+    lib.vp_ce_forward_f32.restype = ctypes.c_int
+    lib.vp_ce_forward_f32.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, i64, i64, vp, sz, vp]
+    lib.vp_ce_backward_f32.restype = ctypes.c_int
+    lib.vp_ce_backward_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, i64, i64,
+                                       ctypes.c_int, vp, sz, vp]
     lib.vp_ce_profile_enable.restype = None
     lib.vp_ce_profile_enable.argtypes = [ctypes.c_int]
     lib.vp_ce_profile_collect.restype = ctypes.c_int
@@ -218,3 +225,37 @@ def vp_ce_forward_static(H, W, labels, block_v: int, ignore_index: int, loss, ls
         int(T_chunk), int(chunk_index_base),
         None if device_status_out is None else _ptr(device_status_out, torch.int32, "device_status_out", 1),
         _stream_ptr(stream)))
+
+
+def vp_ce_workspace_bytes_f32(T_chunk: int, d: int, block_v: int) -> int:
+    return int(load_library().vp_ce_workspace_bytes_f32(int(T_chunk), int(d), int(block_v)))
+
+
+def vp_ce_forward_f32(H, W, labels, block_v: int, ignore_index: int, loss, lse, T_chunk: int,
+                      chunk_index_base: int, workspace, stream=None) -> None:
+    """vp_ce_forward for float32 H and W (TF32 tensor cores)."""
+    import torch
+    lib = load_library()
+    T, d, V = _shapes(H, W)
+    _check(lib.vp_ce_forward_f32(
+        _ptr(H, torch.float32, "H"), _ptr(W, torch.float32, "W"), _ptr(labels, torch.int32, "labels", T),
+        T, d, V, int(block_v), int(ignore_index),
+        _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
+        int(T_chunk), int(chunk_index_base),
+        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+
+
+def vp_ce_backward_f32(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index: int, T_chunk: int,
+                       chunk_index_base: int, accumulate_dW: bool, workspace, stream=None) -> None:
+    """vp_ce_backward for float32 H and W; dH is float32."""
+    import torch
+    lib = load_library()
+    T, d, V = _shapes(H, W)
+    _check(lib.vp_ce_backward_f32(
+        _ptr(H, torch.float32, "H"), _ptr(W, torch.float32, "W"), _ptr(labels, torch.int32, "labels", T),
+        _ptr(lse, torch.float32, "lse", T),
+        None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
+        _ptr(dH, torch.float32, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
+        T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
+        1 if accumulate_dW else 0,
+        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))

@@ -146,6 +146,14 @@ __device__ __forceinline__ void umma2_f16(uint32_t tmem_d, uint64_t adesc, uint6
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same for 32-bit inputs read as TF32 (K = 8 per instruction).
+__device__ __forceinline__ void umma2_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma2_commit_local(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -233,18 +241,22 @@ __device__ __forceinline__ float ex2f(float x) {
 //   K-major operand : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (SBO); LBO unused.
 //   MN-major operand: 64 K-rows of 64 MN elements (128 B) per box; boxes of successive
 //                     64-element MN chunks LBO bytes apart; 8-K-row groups 1024 B apart (SBO).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+//   layout: 2 = 128-byte swizzle in 16-byte units; 1 = 128-byte swizzle in 32-byte units (MN-major operands of
+//   32-bit element types: the tensor core transposes them in 32-byte pieces).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                   uint64_t layout = 2) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
     d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
     d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
     d |= 1ull << 46;                      // descriptor version of sm_100
-    d |= 2ull << 61;                      // SWIZZLE_128B
+    d |= layout << 61;                    // swizzle mode
     return d;
 }
 // Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = m (128, or 256 for a CTA pair), N = bn.
-__host__ __device__ constexpr uint32_t make_idesc(int bn, bool a_mn, bool b_mn, int m) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn) << 15) |
+// fmt: operand format field, 1 = bf16 (kind::f16), 2 = tf32 (kind::tf32).
+__host__ __device__ constexpr uint32_t make_idesc(int bn, bool a_mn, bool b_mn, int m, uint32_t fmt = 1u) {
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(a_mn) << 15) |
            (static_cast<uint32_t>(b_mn) << 16) | (static_cast<uint32_t>(bn >> 3) << 17) |
            (static_cast<uint32_t>(m >> 4) << 24);
 }

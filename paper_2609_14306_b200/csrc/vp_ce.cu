@@ -74,7 +74,7 @@ struct WsLayout {
 };
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-bool ws_layout(int64_t T_chunk, int64_t d, int64_t block_v, WsLayout* L) {
+bool ws_layout(int64_t T_chunk, int64_t d, int64_t block_v, WsLayout* L, int g_elem_bytes = 2) {
     if (T_chunk <= 0 || d <= 0 || block_v <= 0) return false;
     if (T_chunk % BM || block_v % BN_VOCAB || d % 8) return false;
     if (T_chunk > (1 << 24) || block_v > (1 << 24) || d > (1 << 20)) return false;
@@ -88,7 +88,7 @@ bool ws_layout(int64_t T_chunk, int64_t d, int64_t block_v, WsLayout* L) {
     L->ylab = off;    off = align_up(off + 4 * T_chunk, 1024);
     L->pm = off;      off = align_up(off + 4 * T_chunk * nt, 1024);
     L->pz = off;      off = align_up(off + 4 * T_chunk * nt, 1024);
-    L->G = off;       off = align_up(off + 2 * static_cast<size_t>(T_chunk) * block_v, 1024);
+    L->G = off;       off = align_up(off + g_elem_bytes * static_cast<size_t>(T_chunk) * block_v, 1024);
     L->acc = off;     off = align_up(off + 4 * static_cast<size_t>(T_chunk) * d, 1024);
     L->total = off;
     return true;
@@ -107,16 +107,18 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
     return fn;
 }
 
-// 2-D bf16 tensor map over a row-major [rows, cols] matrix: dim0 = cols (contiguous), 128-byte swizzle.
+// 2-D tensor map over a row-major [rows, cols] matrix of bf16 (elem_bytes 2) or fp32 (4): dim0 = cols
+// (contiguous), 128-byte swizzle.
 bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld_elems, uint32_t box_cols,
-              uint32_t box_rows) {
+              uint32_t box_rows, int elem_bytes = 2) {
     auto enc = get_encode();
     if (!enc) return false;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {ld_elems * 2};
+    cuuint64_t strides[1] = {ld_elems * elem_bytes};
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+    const CUtensorMapDataType dt = elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    CUresult r = enc(map, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -125,15 +127,21 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
 // MN-major operand of a row-major [k_rows, mn_cols] matrix (mn_cols % 64 == 0) as a 3-D tensor
 // {64 contiguous elements, k_rows, mn_cols / 64}: one box {64, 64, chunks} per k-block lands in
 // shared memory as `chunks` consecutive 64 x 128-byte blocks, the layout the MMA descriptor expects.
-bool make_map_mn3d(CUtensorMap* map, const void* ptr, uint64_t k_rows, uint64_t mn_cols, uint64_t ld_elems, uint32_t chunks) {
+// (fp32: chunks of 32 elements and 32 k-rows per box.)
+bool make_map_mn3d(CUtensorMap* map, const void* ptr, uint64_t k_rows, uint64_t mn_cols, uint64_t ld_elems, uint32_t chunks,
+                   int elem_bytes = 2) {
     auto enc = get_encode();
-    if (!enc || mn_cols % 64) return false;
-    cuuint64_t dims[3] = {64, k_rows, mn_cols / 64};
-    cuuint64_t strides[2] = {ld_elems * 2, 128};
-    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(BK), chunks};
+    const uint64_t ce = 128 / elem_bytes;                 // elements per 128-byte chunk row = k-rows per stage
+    if (!enc || mn_cols % ce) return false;
+    cuuint64_t dims[3] = {ce, k_rows, mn_cols / ce};
+    cuuint64_t strides[2] = {ld_elems * elem_bytes, 128};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(ce), static_cast<cuuint32_t>(ce), chunks};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    const CUtensorMapDataType dt = elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    // MN-major 32-bit operands are swizzled in 32-byte units (what the tensor core expects for them)
+    const CUtensorMapSwizzle sw = elem_bytes == 4 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
+    CUresult r = enc(map, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -184,11 +192,11 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     return cudaGetLastError();
 }
 
-template <int BN, bool A_MN, bool B_MN, int EPI>
+template <int BN, bool A_MN, bool B_MN, int EPI, bool TF32 = false>
 cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const GemmParams& p,
                         cudaStream_t st) {
     constexpr int SMEM = pair_smem_total<BN, EPI>();
-    auto kern = vpce_gemm_pair_kernel<BN, A_MN, B_MN, EPI>;
+    auto kern = vpce_gemm_pair_kernel<BN, A_MN, B_MN, EPI, TF32>;
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -699,3 +707,5 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
 }
 
 }  // extern "C"
+
+#include "vp_ce_f32.inc"

@@ -190,6 +190,51 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtens
     }
 }
 
+// fp32 variant for the TF32 path: per 32 columns a 32 x 128-byte box of floats.
+__device__ __forceinline__ void epilogue_resid_f32(const GemmParams& p, const CUtensorMap* tmG, uint32_t stage_smem,
+                                                   int mt, int nt, int row, int lane, uint32_t tmem_row) {
+    const int grow = mt * BM + row;
+    const bool row_ok = grow < p.rows_valid;
+    int label = row_ok ? p.labels[grow] : p.ignore_index;
+    const bool valid = row_ok && label != p.ignore_index && static_cast<unsigned>(label) < static_cast<unsigned>(p.V);
+    float dl = 0.f, lseL = 0.f;
+    if (valid) dl = p.dloss ? p.dloss[grow] : *p.inv_n_valid;
+    if (row_ok) lseL = p.lse[grow] * LOG2E;
+    const int lrel = valid ? label - (p.v_lo + nt * BN_VOCAB) : -1;
+    const uint64_t pol_c = make_policy(p.hint_c);
+#pragma unroll 1
+    for (int c = 0; c < BN_VOCAB / 32; ++c) {
+        const uint32_t buf = stage_smem + (c & 1) * 4096;
+        if (lane == 0) bulk_wait_read_1();
+        __syncwarp();
+        float v[32];
+        tmem_ld32(tmem_row + c * 32, v);
+        tmem_ld_wait();
+        const int nvalid = p.cols_valid - (nt * BN_VOCAB + c * 32);
+        const int jj = lrel - c * 32;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            float g = dl * ex2f(fmaf(v[j], LOG2E, -lseL));
+            if (j == jj) g -= dl;
+            v[j] = (j < nvalid) ? g : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint4 o;
+            o.x = __float_as_uint(v[4 * q]); o.y = __float_as_uint(v[4 * q + 1]);
+            o.z = __float_as_uint(v[4 * q + 2]); o.w = __float_as_uint(v[4 * q + 3]);
+            st_shared_v4(buf + lane * 128 + ((q ^ (lane & 7)) << 4), o);
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0 && mt * BM < p.g_rows) {
+            if (p.hint_c) tma_store_2d_hint(tmG, buf, nt * BN_VOCAB + c * 32, mt * BM + (row - lane), pol_c);
+            else tma_store_2d(tmG, buf, nt * BN_VOCAB + c * 32, mt * BM + (row - lane));
+            bulk_commit();
+        }
+    }
+}
+
 // ncol0: first output column of the tile; n_this: its width (columns beyond cols_valid are skipped).
 __device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
     const int grow = mt * BM + row;
@@ -496,7 +541,7 @@ template <int BN, int EPI> constexpr int pair_smem_total() {
     return PairCfg<BN>::SMEM_TOTAL + (EPI == EPI_RESID ? G_STAGING_BYTES : 0);
 }
 
-template <int BN, bool A_MN, bool B_MN, int EPI>
+template <int BN, bool A_MN, bool B_MN, int EPI, bool TF32 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                       const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
@@ -505,6 +550,11 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     constexpr uint32_t TMEM_COLS = 512u;
     constexpr uint32_t ACC_STRIDE = 256u;
     static_assert(BN == 256, "pair tiles are 256 x 256");
+    // Element-size dependent geometry: a 128-byte swizzled row holds BKE elements (one k-block of a K-major
+    // operand, one chunk of an MN-major operand); one MMA consumes UK of them along K.
+    constexpr int BKE = TF32 ? 32 : 64;
+    constexpr int CSH = TF32 ? 5 : 6;
+    constexpr int UK = TF32 ? 8 : 16;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -558,7 +608,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     // of 64 (one swizzled chunk) when B is MN-major.
     auto tile_n = [&](int nt) {
         const int left = p.cols_valid - nt * BN;
-        constexpr int R = B_MN ? 128 : 32;
+        constexpr int R = B_MN ? 2 * BKE : 32;
         return left >= BN ? BN : ((left + R - 1) / R * R);
     };
     // The work list, handed out dynamically (greedy list scheduling):
@@ -646,10 +696,10 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     const uint32_t bar = mapa_shared(full_bar(stage), 0);    // the leader's barrier
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
                     const uint32_t sb = sa + Cfg::A_BYTES;
-                    if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BK, (p.a_mn0 + mt * BM) >> 6, pol_a);
-                    else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BK, p.a_mn0 + mt * BM, pol_a);
-                    if (B_MN) tma2_load_3d(sb, &tmB, bar, 0, p.b_k0 + kb * BK, (p.b_mn0 + bn0) >> 6, pol_b);
-                    else tma2_load_2d(sb, &tmB, bar, p.b_k0 + kb * BK, p.b_mn0 + bn0, pol_b);
+                    if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BKE, (p.a_mn0 + mt * BM) >> CSH, pol_a);
+                    else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BKE, p.a_mn0 + mt * BM, pol_a);
+                    if (B_MN) tma2_load_3d(sb, &tmB, bar, 0, p.b_k0 + kb * BKE, (p.b_mn0 + bn0) >> CSH, pol_b);
+                    else tma2_load_2d(sb, &tmB, bar, p.b_k0 + kb * BKE, p.b_mn0 + bn0, pol_b);
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -679,7 +729,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 int pmt, nt, ncol0, width;
                 get_tile(tile, pmt, nt, ncol0, width);
                 if (width == 0) continue;
-                const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM);
+                const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM, TF32 ? 2u : 1u);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
                 if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
@@ -690,13 +740,18 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     tc_fence_after();
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
                     const uint32_t sb = sa + Cfg::A_BYTES;
-                    const uint64_t adesc = A_MN ? make_smem_desc(sa, BK * 128, 1024) : make_smem_desc(sa, 16, 1024);
-                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, BK * 128, 1024) : make_smem_desc(sb, 16, 1024);
+                    // MN-major 32-bit operands: 32-byte swizzle units, whose pattern repeats every 4 k-rows (512 B)
+                    constexpr uint64_t MN_LAYOUT = TF32 ? 1 : 2;
+                    constexpr uint32_t MN_SBO = TF32 ? 512 : 1024;
+                    const uint64_t adesc = A_MN ? make_smem_desc(sa, BKE * 128, MN_SBO, MN_LAYOUT) : make_smem_desc(sa, 16, 1024);
+                    const uint64_t bdesc = B_MN ? make_smem_desc(sb, BKE * 128, MN_SBO, MN_LAYOUT) : make_smem_desc(sb, 16, 1024);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
-                        umma2_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < BKE / UK; ++k) {
+                        // K-major: UK elements = 32 B along the swizzled row; MN-major: UK k-rows of 128 B
+                        const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UK * 128 : k * 32) >> 4);
+                        const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UK * 128 : k * 32) >> 4);
+                        if (TF32) umma2_tf32(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
+                        else umma2_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     umma2_commit_both(empty_bar(stage));                     // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -737,6 +792,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             tc_fence_after();
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
+            else if (EPI == EPI_RESID && TF32) epilogue_resid_f32(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
             else if (EPI == EPI_DH) epilogue_dh(p, mt, ncol0, row, tmem_row, width);
             else epilogue_dw(p, mt, ncol0, row, tmem_row, width);

@@ -189,6 +189,47 @@ def gaussian_bf16(shape, std: float, seed: int, stream: int, call_index: int = 0
     return out
 
 
+def f32_round_to_tf32(x: np.ndarray) -> np.ndarray:
+    """Round float32 to the nearest value with a 10-bit mantissa (TF32), ties to even; result is float32."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + (np.uint32(0xFFF) + ((u >> np.uint32(13)) & np.uint32(1)))) & np.uint32(0xFFFFE000)
+    return r.view(np.float32)
+
+
+def gaussian_f32(shape, std: float, seed: int, stream: int, call_index: int = 0, tf32: bool = True) -> np.ndarray:
+    """N(0, std^2) float32 draws, same slab/seed scheme as gaussian_bf16; inputs of the FP32 (TF32 tensor
+    core) entry points.  With ``tf32`` (default) the draws are rounded to TF32-representable values, so that
+    the tensor core's products are exact and the float64 oracle sees the very numbers the GPU multiplies
+    (the counterpart of rounding the bf16 path's inputs to bf16)."""
+    rows, cols = int(shape[0]), int(shape[1])
+    out = np.empty((rows, cols), dtype=np.float32)
+    s = np.float32(std)
+
+    def fill(k: int) -> None:
+        r0, r1 = k * SLAB_ROWS, min(rows, (k + 1) * SLAB_ROWS)
+        rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, stream, call_index, k])))
+        x = rng.standard_normal((r1 - r0, cols), dtype=np.float32)
+        if std != 1.0:
+            x *= s
+        out[r0:r1] = f32_round_to_tf32(x) if tf32 else x
+
+    n_slabs = -(-rows // SLAB_ROWS)
+    if n_slabs == 1:
+        fill(0)
+    else:
+        with ThreadPoolExecutor(_threads()) as ex:
+            list(ex.map(fill, range(n_slabs)))
+    return out
+
+
+def make_weights_f32(w: Workload, tf32: bool = True) -> np.ndarray:
+    return gaussian_f32((w.V, w.d), w.w_std, w.seed, STREAM_W, 0, tf32)
+
+
+def make_hidden_f32(w: Workload, call_index: int = 0, tf32: bool = True) -> np.ndarray:
+    return gaussian_f32((w.T, w.d), 1.0, w.seed, STREAM_H, call_index, tf32)
+
+
 def zipf_cdf(V: int, s: float) -> np.ndarray:
     """CDF of the Zipf law truncated to ranks 1..V, p(k) proportional to k^-s (float64)."""
     p = np.arange(1, V + 1, dtype=np.float64) ** (-float(s))
