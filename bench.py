@@ -184,6 +184,8 @@ def main():
     ap.add_argument("--t-chunk", type=int, default=0)
     ap.add_argument("--shape", default="", help="custom workload T,d,V,block_v (Gaussian inputs, Zipf labels); "
                                                 "for kernel experiments, not a benchmark config")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "tf32"],
+                    help="bf16 inputs (the benchmark's metric) or float32 inputs on TF32 tensor cores (the paper's precision)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-in-timed-region", type=int, default=1)
@@ -222,27 +224,35 @@ def main():
     chunks_per_call = -(-w.T // T_chunk)
 
     # ---- inputs (host, seeded) -> device.  Each rank of a multi-GPU run draws its own batch stream.
-    W_bits = make_weights(w)
+    tf32 = args.dtype == "tf32"
+    if tf32:
+        from synth_inputs import make_hidden_f32, make_weights_f32
+        make_w, make_h = make_weights_f32, make_hidden_f32
+        to_dev = lambda a: torch.from_numpy(a).to(dev)
+        fwd, bwd, ws_fn = vp.vp_ce_forward_f32, vp.vp_ce_backward_f32, vp.vp_ce_workspace_bytes_f32
+    else:
+        make_w, make_h = make_weights, make_hidden
+        to_dev = lambda bits: torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+        fwd, bwd, ws_fn = vp.vp_ce_forward, vp.vp_ce_backward, vp.vp_ce_workspace_bytes
+    W_bits = make_w(w)
     labels_all = stream_labels(w)
-    def bf16_dev(bits):
-        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
-    Wd = bf16_dev(W_bits)
-    H_host0 = make_hidden(w, 0) if rank == 0 else None
+    Wd = to_dev(W_bits)
+    H_host0 = make_h(w, 0) if rank == 0 else None
     Hs, labs = [], []
     for call in range(w.n_calls):
-        hb = H_host0 if (call == 0 and rank == 0) else make_hidden(rank_workload(w, rank), call)
-        Hs.append(bf16_dev(hb))
+        hb = H_host0 if (call == 0 and rank == 0) else make_h(rank_workload(w, rank), call)
+        Hs.append(to_dev(hb))
         labs.append(torch.from_numpy(labels_all[call * w.T:(call + 1) * w.T].copy()).to(dev))
     n_valid_total = int((labels_all != IGNORE_INDEX).sum())
 
     torch.cuda.synchronize()
     resident = torch.cuda.memory_allocated(dev)
     torch.cuda.reset_peak_memory_stats(dev)
-    ws_bytes = vp.vp_ce_workspace_bytes(T_chunk, w.d, w.block_v)
+    ws_bytes = ws_fn(T_chunk, w.d, w.block_v)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     loss = [torch.empty(w.T, dtype=torch.float32, device=dev) for _ in range(w.n_calls)]
     lse = [torch.empty(w.T, dtype=torch.float32, device=dev) for _ in range(w.n_calls)]
-    dH = [torch.empty(w.T, w.d, dtype=torch.bfloat16, device=dev) for _ in range(w.n_calls)]
+    dH = [torch.empty(w.T, w.d, dtype=torch.float32 if tf32 else torch.bfloat16, device=dev) for _ in range(w.n_calls)]
     dW = torch.empty(w.V, w.d, dtype=torch.float32, device=dev)
     mean = torch.zeros(1, dtype=torch.float32, device=dev)
     nval = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -257,9 +267,9 @@ def main():
         step_no[0] += 1
         for call in range(w.n_calls):
             base = (call + step_no[0]) * chunks_per_call
-            vp.vp_ce_forward(Hs[call], Wd, labs[call], w.block_v, IGNORE_INDEX, loss[call], lse[call], T_chunk, base, ws)
-            vp.vp_ce_backward(Hs[call], Wd, labs[call], lse[call], None if dl_stream is None else dl_stream[call],
-                              dH[call], dW, w.block_v, IGNORE_INDEX, T_chunk, base, call > 0, ws)
+            fwd(Hs[call], Wd, labs[call], w.block_v, IGNORE_INDEX, loss[call], lse[call], T_chunk, base, ws)
+            bwd(Hs[call], Wd, labs[call], lse[call], None if dl_stream is None else dl_stream[call],
+                dH[call], dW, w.block_v, IGNORE_INDEX, T_chunk, base, call > 0, ws)
             vp.vp_ce_mean_loss(loss[call], labs[call], w.V, IGNORE_INDEX, mean, nval)
 
     def barrier():
@@ -309,7 +319,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point
     e2e = None
-    if not args.no_e2e and w.n_calls == 1:
+    if not args.no_e2e and w.n_calls == 1 and not tf32:
         Hh = torch.empty(w.T, w.d, dtype=torch.bfloat16).pin_memory()
         Hh.copy_(Hs[0].cpu())
         lh = labs[0].cpu().pin_memory()
@@ -338,13 +348,19 @@ def main():
         return
 
     peaks, peak_src = load_peaks()
+    if tf32:
+        # no TF32 peak is measured on this machine: the measured bf16 peaks times the nominal dense ratio (1.1 / 2.25 PFLOP/s)
+        ratio = 1100.0 / NOMINAL_BF16_TFLOPS
+        peaks = dict(peaks, bf16_tflops=peaks["bf16_tflops"] * ratio,
+                     bf16_tflops_sustained=peaks["bf16_tflops_sustained"] * ratio)
+        peak_src += " bf16 peak x nominal tf32/bf16 ratio 0.489"
     tokens = w.T_stream
     value = whole_job_tokens_per_s(world, tokens, ms_step)
     tflops = w.flops / (ms_step / 1e3) / 1e12
     out = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
         "config": {"workload": w.name, "T": w.T, "calls_per_step": w.n_calls, "d": w.d, "V": w.V,
                    "block_v": w.block_v, "T_chunk": T_chunk, "P": w.P, "ignored_labels": w.n_ignored,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
@@ -352,10 +368,10 @@ def main():
         "tflops_per_gpu": tflops,
         "frac_of_bf16_peak": {"burst_measured": tflops / peaks["bf16_tflops"],
                               "sustained_measured": tflops / peaks["bf16_tflops_sustained"],
-                              "nominal_2250": tflops / NOMINAL_BF16_TFLOPS, "source": peak_src},
+                              "nominal_2250": tflops / (1100.0 if tf32 else NOMINAL_BF16_TFLOPS), "source": peak_src},
         "flops_per_step": w.flops,
         "peak_bytes": {"workspace_bytes": ws_bytes, "increment_over_resident_inputs": int(peak_extra),
-                       "outputs_bytes": int(w.T_stream * 8 + w.T_stream * w.d * 2 + w.V * w.d * 4),
+                       "outputs_bytes": int(w.T_stream * 8 + w.T_stream * w.d * (4 if tf32 else 2) + w.V * w.d * 4),
                        "full_fp32_logits_bytes": w.logits_bytes_fp32,
                        "dense_fwd_bwd_would_hold_bytes": 3 * w.logits_bytes_fp32},
         "mean_loss": mean_loss, "device_status": status,
@@ -381,12 +397,12 @@ def main():
                            "flops_per_launch": flops_kind / kinds[dom]["launches"],
                            "avg_launch_ms": kinds[dom]["avg_ms"],
                            "traffic": (NCU_DRAM_BYTES_PER_LAUNCH[dom]
-                                       if (w.d, w.block_v, T_chunk) == (2880, 8192, 16384) else None),
+                                       if (w.d, w.block_v, T_chunk) == (2880, 8192, 16384) and not tf32 else None),
                            "traffic_unit": "bytes of DRAM per launch (ncu)"}
         out["kernels"] = kinds
     if e2e:
         out["e2e"] = e2e
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and not tf32:
         hb = H_host0
         cb, _, _ = oracle_sample_rate(w, W_bits, hb, labels_all[:w.T])
         out["cpu_baseline"] = cb

@@ -113,6 +113,8 @@ PROFILE_WORKLOADS: Dict[str, Workload] = {
         # The shape of the paper's isolated Ring-DTP benchmark (App. C: N = 16384 tokens per GPU, H = 7168,
         # V = 200000, P = 8), for a context line beside its Table 2; V/P = 25000 is rounded up to the next
         # multiple of the 256-column tile.  The paper runs it in FP32, this build in bf16.
+        Workload("papershape32k", T=32768, d=7168, V=200000, block_v=25088, T_chunk=32768,
+                 w_std=0.006, labels="zipf", zipf_s=1.1, ignore_frac=0.0, seed=15),
         Workload("papershape", T=16384, d=7168, V=200000, block_v=25088, T_chunk=16384,
                  w_std=0.006, labels="zipf", zipf_s=1.1, ignore_frac=0.0, seed=14),
     ]
