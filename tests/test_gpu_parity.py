@@ -258,3 +258,48 @@ def test_large_logits_stay_finite_and_accurate():
     # fp32 logits of this size carry ~1e-5 relative error, so compare relatively
     assert np.abs(run.np_lse() - ref["lse"]).max() <= 2e-5 * np.abs(ref["lse"]).max() + TOL_TOKEN
     assert relF(run.np_dH(), ref["dH"]) <= TOL_GRAD and relF(run.np_dW(), ref["dW"]) <= TOL_GRAD
+
+
+def test_host_buffer_entry_point_matches_oracle():
+    """vp_ce_fwd_bwd_host: activations in pinned host memory, copies inside the call."""
+    w = custom_workload("host", T=640, d=256, V=3000, block_v=1024, T_chunk=256, w_std=0.0625,
+                        labels="zipf", ignore_frac=0.1, seed=41)
+    b = make_batch(w)
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    ref = orc.forward_backward(H64, W64, b.labels)
+    Hh = torch.from_numpy(b.H_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    lh = torch.from_numpy(b.labels).pin_memory()
+    Wd = torch.from_numpy(b.W_bits.view(np.int16)).cuda().view(torch.bfloat16)
+    loss_h = torch.full((w.T,), float("nan")).pin_memory()
+    dH_h = torch.zeros(w.T, w.d, dtype=torch.bfloat16).pin_memory()
+    dW = torch.full((w.V, w.d), float("nan"), device="cuda")
+    H_dev = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+    lab_dev = torch.empty(w.T, dtype=torch.int32, device="cuda")
+    loss_dev = torch.empty(w.T, device="cuda")
+    lse_dev = torch.empty(w.T, device="cuda")
+    dH_dev = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(vp.vp_ce_workspace_bytes(w.T_chunk, w.d, w.block_v), dtype=torch.uint8, device="cuda")
+    vp.vp_ce_fwd_bwd_host(Hh, lh, Wd, loss_h, dH_h, dW, w.block_v, IGNORE_INDEX, w.T_chunk, 0, False,
+                          H_dev, lab_dev, loss_dev, lse_dev, dH_dev, ws)
+    # the call synchronises its stream: the host buffers are valid now
+    assert np.abs(loss_h.numpy().astype(np.float64) - ref["loss"]).max() <= TOL_TOKEN
+    assert relF(dH_h.float().numpy().astype(np.float64), ref["dH"]) <= TOL_GRAD
+    assert relF(dW.cpu().numpy().astype(np.float64), ref["dW"]) <= TOL_GRAD
+    assert vp.vp_ce_device_status(ws) == 0
+
+
+def test_profile_hooks_count_launches_per_kernel_kind():
+    w = custom_workload("prof", T=512, d=256, V=2048, block_v=512, T_chunk=256, w_std=0.0625, seed=43)
+    b = make_batch(w)
+    r = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk)
+    n0 = vp.vp_ce_launch_count()
+    vp.vp_ce_profile_enable(True)
+    r.forward().backward()
+    vp.vp_ce_profile_enable(False)
+    stats = vp.vp_ce_profile_collect()
+    meetings = (w.T // w.T_chunk) * w.P                       # one launch of every kind per (chunk, shard)
+    for kind in vp.KERNEL_KINDS:
+        ms, n = stats[kind]
+        assert n == meetings and ms > 0.0
+    assert vp.vp_ce_launch_count() - n0 >= 4 * meetings
+    assert all(n == 0 for _, n in vp.vp_ce_profile_collect().values())     # collected entries are forgotten
