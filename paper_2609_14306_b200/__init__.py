@@ -23,3 +23,11 @@ from .binding import (  # noqa: F401
     vp_ce_status_string,
     vp_ce_workspace_bytes,
 )
+
+
+def __getattr__(name):
+    # the autograd front end needs torch; import it lazily so the C-ABI binding works without it
+    if name in ("vocab_proj_cross_entropy", "vocab_proj_cross_entropy_mean"):
+        from . import autograd as _ag
+        return getattr(_ag, name)
+    raise AttributeError(name)

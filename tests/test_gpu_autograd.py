@@ -1,0 +1,52 @@
+"""The torch.autograd front end against plain PyTorch float32 cross-entropy of the same operation and
+against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_14306_b200 as vp
+from oracle import vpce_oracle as orc
+from synth_inputs import IGNORE_INDEX, bf16_bits_to_f64, custom_workload, make_batch
+from vpce_testlib import TOL_GRAD, TOL_TOKEN, relF, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def test_autograd_mean_loss_matches_pytorch_and_oracle():
+    w = custom_workload("ag", T=640, d=256, V=5000, block_v=1024, T_chunk=256, w_std=0.0625,
+                        labels="zipf", ignore_frac=0.1, seed=51)
+    b = make_batch(w)
+    H = to_dev_bf16(b.H_bits).requires_grad_(True)
+    W = to_dev_bf16(b.W_bits).requires_grad_(True)
+    lab = torch.from_numpy(b.labels).cuda()
+    loss = vp.vocab_proj_cross_entropy_mean(H, W, lab, block_v=w.block_v, T_chunk=w.T_chunk)
+    loss.backward()
+    # plain PyTorch fp32 reference of the same op on the same bf16 values
+    Hr = H.detach().float().requires_grad_(True)
+    Wr = W.detach().float().requires_grad_(True)
+    ref = torch.nn.functional.cross_entropy(Hr @ Wr.T, lab.long(), ignore_index=IGNORE_INDEX)
+    ref.backward()
+    assert abs(loss.item() - ref.item()) <= 1e-4 * abs(ref.item())
+    assert relF(H.grad.float().cpu().numpy(), Hr.grad.cpu().numpy().astype(np.float64)) <= TOL_GRAD
+    assert relF(W.grad.float().cpu().numpy(), Wr.grad.cpu().numpy().astype(np.float64)) <= TOL_GRAD
+    o = orc.forward_backward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), b.labels)
+    assert abs(loss.item() - o["mean"]) <= 1e-4 * abs(o["mean"])
+    assert relF(H.grad.float().cpu().numpy(), o["dH"]) <= TOL_GRAD
+
+
+def test_autograd_per_token_loss_with_fp32_accumulation_buffer():
+    w = custom_workload("ag2", T=384, d=128, V=2000, block_v=512, T_chunk=128, w_std=0.09,
+                        labels="uniform", ignore_frac=0.05, seed=52)
+    b = make_batch(w)
+    H = to_dev_bf16(b.H_bits).requires_grad_(True)
+    W = to_dev_bf16(b.W_bits).requires_grad_(True)
+    lab = torch.from_numpy(b.labels).cuda()
+    dl = np.random.default_rng(0).random(w.T).astype(np.float32)
+    main_grad = torch.zeros(w.V, w.d, dtype=torch.float32, device="cuda")
+    per_tok = vp.vocab_proj_cross_entropy(H, W, lab, block_v=w.block_v, T_chunk=w.T_chunk, dW_accum=main_grad)
+    (per_tok * torch.from_numpy(dl).cuda()).sum().backward()
+    o = orc.forward_backward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), b.labels, dl.astype(np.float64))
+    assert np.abs(per_tok.detach().cpu().numpy() - o["loss"]).max() <= TOL_TOKEN
+    assert W.grad is None                                     # the weight gradient went to the fp32 buffer
+    assert relF(main_grad.cpu().numpy(), o["dW"]) <= TOL_GRAD
+    assert relF(H.grad.float().cpu().numpy(), o["dH"]) <= TOL_GRAD
