@@ -529,7 +529,10 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // Signalling: TMA byte counts of both CTAs are credited to the leader's "full" barrier
 // (.cta_group::2 loads, no multicast); tcgen05.commit with a CTA mask releases the stage in both
 // CTAs and publishes the accumulator to both epilogues; epilogue warps of both CTAs arrive on the
-// leader's "accumulator free" barrier.  Tiles are assigned round-robin to the pairs.
+// leader's "accumulator free" barrier.  Work is handed out dynamically: the leader takes list positions
+// from the launch's counter and publishes them to both CTAs through a small ring (see below).
+// With TF32 = true the operands are 32-bit floats multiplied as TF32 (kind::tf32, K = 8 per MMA,
+// k-blocks of 32 elements); the 128-byte rows and hence all byte sizes are the same.
 template <int BN> struct PairCfg {
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (BN / 2) * BK * 2;
