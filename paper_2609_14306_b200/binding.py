@@ -94,10 +94,28 @@ def vp_ce_workspace_bytes(T_chunk: int, d: int, block_v: int) -> int:
     return int(load_library().vp_ce_workspace_bytes(int(T_chunk), int(d), int(block_v)))
 
 
-def _stream_ptr(stream) -> int:
+def _stream_ptr(stream, like=None) -> int:
+    """Raw cudaStream_t: the given stream, else the current stream of the device that holds `like`."""
     import torch
-    s = torch.cuda.current_stream() if stream is None else stream
-    return int(s.cuda_stream)
+    if stream is not None:
+        return int(stream.cuda_stream)
+    dev = like.device if like is not None else None
+    return int(torch.cuda.current_stream(dev).cuda_stream)
+
+
+class _on_device:
+    """Makes the device that holds the operands current for the duration of a call (the library launches
+    on the current device)."""
+
+    def __init__(self, t):
+        import torch
+        self._guard = torch.cuda.device(t.device)
+
+    def __enter__(self):
+        return self._guard.__enter__()
+
+    def __exit__(self, *a):
+        return self._guard.__exit__(*a)
 
 
 def _ptr(t, dtype, name: str, numel: Optional[int] = None) -> int:
@@ -125,12 +143,13 @@ def vp_ce_forward(H, W, labels, block_v: int, ignore_index: int, loss, lse, T_ch
     import torch
     lib = load_library()
     T, d, V = _shapes(H, W)
-    _check(lib.vp_ce_forward(
-        _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
-        T, d, V, int(block_v), int(ignore_index),
-        _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
-        int(T_chunk), int(chunk_index_base),
-        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+    with _on_device(H):
+        _check(lib.vp_ce_forward(
+            _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
+            T, d, V, int(block_v), int(ignore_index),
+            _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
+            int(T_chunk), int(chunk_index_base),
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
 
 
 def vp_ce_backward(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index: int, T_chunk: int,
@@ -139,31 +158,35 @@ def vp_ce_backward(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index:
     import torch
     lib = load_library()
     T, d, V = _shapes(H, W)
-    _check(lib.vp_ce_backward(
-        _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
-        _ptr(lse, torch.float32, "lse", T),
-        None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
-        _ptr(dH, torch.bfloat16, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
-        T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
-        1 if accumulate_dW else 0,
-        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+    with _on_device(H):
+        _check(lib.vp_ce_backward(
+            _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
+            _ptr(lse, torch.float32, "lse", T),
+            None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
+            _ptr(dH, torch.bfloat16, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
+            T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
+            1 if accumulate_dW else 0,
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
 
 
 def vp_ce_mean_loss(loss, labels, V: int, ignore_index: int, mean_out, n_valid_out, stream=None) -> None:
     import torch
     lib = load_library()
     T = loss.numel()
-    _check(lib.vp_ce_mean_loss(
-        _ptr(loss, torch.float32, "loss"), _ptr(labels, torch.int32, "labels", T), T, int(V), int(ignore_index),
-        _ptr(mean_out, torch.float32, "mean_out", 1), _ptr(n_valid_out, torch.int32, "n_valid_out", 1),
-        _stream_ptr(stream)))
+    with _on_device(loss):
+        _check(lib.vp_ce_mean_loss(
+            _ptr(loss, torch.float32, "loss"), _ptr(labels, torch.int32, "labels", T), T, int(V), int(ignore_index),
+            _ptr(mean_out, torch.float32, "mean_out", 1), _ptr(n_valid_out, torch.int32, "n_valid_out", 1),
+            _stream_ptr(stream, loss)))
 
 
 def vp_ce_device_status(workspace, stream=None) -> int:
     import torch
     lib = load_library()
     out = ctypes.c_int32(-1)
-    _check(lib.vp_ce_device_status(_ptr(workspace, torch.uint8, "workspace"), ctypes.byref(out), _stream_ptr(stream)))
+    with _on_device(workspace):
+        _check(lib.vp_ce_device_status(_ptr(workspace, torch.uint8, "workspace"), ctypes.byref(out),
+                                       _stream_ptr(stream, workspace)))
     return int(out.value)
 
 
@@ -184,15 +207,16 @@ def vp_ce_fwd_bwd_host(H_host, labels_host, W, loss_host, dH_host, dW, block_v: 
     lib = load_library()
     T, d = int(H_host.shape[0]), int(H_host.shape[1])
     V = int(W.shape[0])
-    _check(lib.vp_ce_fwd_bwd_host(
-        _host_ptr(H_host, torch.bfloat16, "H_host", T * d), _host_ptr(labels_host, torch.int32, "labels_host", T),
-        _ptr(W, torch.bfloat16, "W", V * d), _host_ptr(loss_host, torch.float32, "loss_host", T),
-        _host_ptr(dH_host, torch.bfloat16, "dH_host", T * d), _ptr(dW, torch.float32, "dW", V * d),
-        T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base), 1 if accumulate_dW else 0,
-        _ptr(H_dev, torch.bfloat16, "H_dev", T * d), _ptr(labels_dev, torch.int32, "labels_dev", T),
-        _ptr(loss_dev, torch.float32, "loss_dev", T), _ptr(lse_dev, torch.float32, "lse_dev", T),
-        _ptr(dH_dev, torch.bfloat16, "dH_dev", T * d),
-        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+    with _on_device(W):
+        _check(lib.vp_ce_fwd_bwd_host(
+            _host_ptr(H_host, torch.bfloat16, "H_host", T * d), _host_ptr(labels_host, torch.int32, "labels_host", T),
+            _ptr(W, torch.bfloat16, "W", V * d), _host_ptr(loss_host, torch.float32, "loss_host", T),
+            _host_ptr(dH_host, torch.bfloat16, "dH_host", T * d), _ptr(dW, torch.float32, "dW", V * d),
+            T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base), 1 if accumulate_dW else 0,
+            _ptr(H_dev, torch.bfloat16, "H_dev", T * d), _ptr(labels_dev, torch.int32, "labels_dev", T),
+            _ptr(loss_dev, torch.float32, "loss_dev", T), _ptr(lse_dev, torch.float32, "lse_dev", T),
+            _ptr(dH_dev, torch.bfloat16, "dH_dev", T * d),
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, W)))
 
 
 KERNEL_KINDS = ("fwd_strip_fold", "bwd_strip_residual", "dH_gemm", "dW_gemm")
@@ -218,13 +242,14 @@ def vp_ce_forward_static(H, W, labels, block_v: int, ignore_index: int, loss, ls
     import torch
     lib = load_library()
     T, d, V = _shapes(H, W)
-    _check(lib.vp_ce_forward_static(
-        _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
-        T, d, V, int(block_v), int(ignore_index),
-        _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
-        int(T_chunk), int(chunk_index_base),
-        None if device_status_out is None else _ptr(device_status_out, torch.int32, "device_status_out", 1),
-        _stream_ptr(stream)))
+    with _on_device(H):
+        _check(lib.vp_ce_forward_static(
+            _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
+            T, d, V, int(block_v), int(ignore_index),
+            _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
+            int(T_chunk), int(chunk_index_base),
+            None if device_status_out is None else _ptr(device_status_out, torch.int32, "device_status_out", 1),
+            _stream_ptr(stream, H)))
 
 
 def vp_ce_workspace_bytes_f32(T_chunk: int, d: int, block_v: int) -> int:
@@ -237,12 +262,13 @@ def vp_ce_forward_f32(H, W, labels, block_v: int, ignore_index: int, loss, lse, 
     import torch
     lib = load_library()
     T, d, V = _shapes(H, W)
-    _check(lib.vp_ce_forward_f32(
-        _ptr(H, torch.float32, "H"), _ptr(W, torch.float32, "W"), _ptr(labels, torch.int32, "labels", T),
-        T, d, V, int(block_v), int(ignore_index),
-        _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
-        int(T_chunk), int(chunk_index_base),
-        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+    with _on_device(H):
+        _check(lib.vp_ce_forward_f32(
+            _ptr(H, torch.float32, "H"), _ptr(W, torch.float32, "W"), _ptr(labels, torch.int32, "labels", T),
+            T, d, V, int(block_v), int(ignore_index),
+            _ptr(loss, torch.float32, "loss", T), _ptr(lse, torch.float32, "lse", T),
+            int(T_chunk), int(chunk_index_base),
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
 
 
 def vp_ce_backward_f32(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index: int, T_chunk: int,
@@ -251,11 +277,12 @@ def vp_ce_backward_f32(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_in
     import torch
     lib = load_library()
     T, d, V = _shapes(H, W)
-    _check(lib.vp_ce_backward_f32(
-        _ptr(H, torch.float32, "H"), _ptr(W, torch.float32, "W"), _ptr(labels, torch.int32, "labels", T),
-        _ptr(lse, torch.float32, "lse", T),
-        None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
-        _ptr(dH, torch.float32, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
-        T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
-        1 if accumulate_dW else 0,
-        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream)))
+    with _on_device(H):
+        _check(lib.vp_ce_backward_f32(
+            _ptr(H, torch.float32, "H"), _ptr(W, torch.float32, "W"), _ptr(labels, torch.int32, "labels", T),
+            _ptr(lse, torch.float32, "lse", T),
+            None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
+            _ptr(dH, torch.float32, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
+            T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
+            1 if accumulate_dW else 0,
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
