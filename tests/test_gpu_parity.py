@@ -41,6 +41,7 @@ def test_config2_mid():
     (257, 40, 300, 256, 128),       # tiny d (one partial K block), T = 2 tiles + 1 row
     (512, 2880, 2048, 512, 256),    # d = 2880 selects the 192-column gradient tile
     (384, 512, 5000, 1024, 384),    # T_chunk of three tiles, 5 shards, last one ragged
+    (200, 64, 600, 512, 1024),      # T_chunk larger than the batch: one short chunk
 ])
 def test_ragged_shapes(T, d, V, block_v, T_chunk):
     w = custom_workload(f"r{T}x{d}x{V}", T=T, d=d, V=V, block_v=block_v, T_chunk=T_chunk,
