@@ -533,22 +533,24 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // from the launch's counter and publishes them to both CTAs through a small ring (see below).
 // With TF32 = true the operands are 32-bit floats multiplied as TF32 (kind::tf32, K = 8 per MMA,
 // k-blocks of 32 elements); the 128-byte rows and hence all byte sizes are the same.
-template <int BN> struct PairCfg {
+// The residual kernel gives 32 KB of the 227 KB to its store staging; the others use them for a 7th stage.
+template <int BN, int EPI = EPI_RESID> struct PairCfg {
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (BN / 2) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
+    static constexpr int BUDGET = SMEM_BUDGET + (EPI == EPI_RESID ? 0 : 28 * 1024);
+    static constexpr int STAGES = (BUDGET / STAGE_BYTES) > 8 ? 8 : (BUDGET / STAGE_BYTES);
     static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
 };
 template <int BN, int EPI> constexpr int pair_smem_total() {
-    return PairCfg<BN>::SMEM_TOTAL + (EPI == EPI_RESID ? G_STAGING_BYTES : 0);
+    return PairCfg<BN, EPI>::SMEM_TOTAL + (EPI == EPI_RESID ? G_STAGING_BYTES : 0);
 }
 
 template <int BN, bool A_MN, bool B_MN, int EPI, bool TF32 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                       const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-    using Cfg = PairCfg<BN>;
+    using Cfg = PairCfg<BN, EPI>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr uint32_t TMEM_COLS = 512u;
     constexpr uint32_t ACC_STRIDE = 256u;
