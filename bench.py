@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
 # profiles/gemm_kernels_moe120b_launch_geometry.md; valid for launches of T_chunk=16384 x block_v=8192 at d=2880.
-NCU_DRAM_BYTES_PER_LAUNCH = {"fwd_strip_fold": 157e6, "bwd_strip_residual": 478e6, "dH_gemm": 891e6, "dW_gemm": 979e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"fwd_strip_fold": 156e6, "bwd_strip_residual": 462e6, "dH_gemm": 776e6, "dW_gemm": 964e6}
 # Token chunk used by the timed launch configuration (a call argument of the library).
 BENCH_T_CHUNK = {"tiny": 512, "mid": 4096, "moe120b": 16384, "moe667b": 8192, "longctx": 16384}
 
