@@ -84,6 +84,8 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels,
  * the masked mean (1 / n_valid on valid tokens, n_valid counted from labels; 0 valid tokens
  * give zero gradients).  dH is overwritten.  dW is overwritten when accumulate_dW == 0 and
  * added to otherwise (fp32 accumulation across calls of a streamed context).
+ * Either dH or dW (not both) may be NULL: that gradient and its contraction are skipped
+ * (a frozen projection weight, or an input that needs no gradient).
  */
 vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse,
                            const float* dloss, void* dH, float* dW,
@@ -96,14 +98,27 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
  * per-token values; this is the reduction the benchmark's metric is stated on).
  * mean_out[0] = sum of loss over valid tokens / n_valid (0 when n_valid == 0);
  * n_valid_out[0] = n_valid.  Both are device pointers.  Deterministic (fixed order).
+ * T == 0 is accepted (mean 0, n_valid 0; loss and labels may then be NULL).
  */
 vpce_status vp_ce_mean_loss(const float* loss, const int32_t* labels, int64_t T, int64_t V,
                             int32_t ignore_index, float* mean_out, int32_t* n_valid_out, void* stream);
 
 /*
+ * Gradient of that masked mean with respect to the per-token loss (chain rule for callers that
+ * differentiate through vp_ce_mean_loss; not in the paper): dloss_out[n] = upstream / n_valid for
+ * valid tokens and 0 for the others.  n_valid is the DEVICE int32 that vp_ce_mean_loss wrote,
+ * upstream a DEVICE float (NULL means 1).  n_valid == 0 gives all zeros.  T == 0 launches nothing.
+ */
+vpce_status vp_ce_mean_loss_grad(const int32_t* labels, int64_t T, int64_t V, int32_t ignore_index,
+                                 const int32_t* n_valid, const float* upstream, float* dloss_out, void* stream);
+
+/*
  * Copies the device status word of `workspace` to host_out[0] (HOST pointer) and
  * synchronises `stream`.  0 means no device-side condition was seen since the last
- * vp_ce_forward / vp_ce_backward call on this workspace began.
+ * vp_ce_forward / vp_ce_backward call on this workspace began: each of those two calls clears the
+ * word first, so a caller that runs them back to back and wants the forward's conditions reads the
+ * word in between.  vp_ce_fwd_bwd_host clears it once, before its forward half, and the word read
+ * after it covers the whole pass.  Both passes flag a label outside [0, V).
  */
 vpce_status vp_ce_device_status(const void* workspace, int32_t* host_out, void* stream);
 

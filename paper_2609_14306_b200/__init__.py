@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     KERNEL_KINDS,
     vp_ce_launch_count,
     vp_ce_mean_loss,
+    vp_ce_mean_loss_grad,
     vp_ce_status_string,
     vp_ce_workspace_bytes,
 )

@@ -32,15 +32,12 @@ class _VocabProjCE(torch.autograd.Function):
         labels = labels.to(torch.int32).contiguous()
         T, d = H.shape
         T_chunk = _pick_chunk(T, T_chunk)
-        ws = torch.empty(_b.vp_ce_workspace_bytes(T_chunk, d, block_v), dtype=torch.uint8, device=H.device)
-        if ws.numel() == 0:
-            raise ValueError("unsupported shape: d % 8, block_v % 256 or T_chunk % 128")
+        ws = _workspace(T_chunk, d, block_v, H.device)
         loss = torch.empty(T, dtype=torch.float32, device=H.device)
         lse = torch.empty(T, dtype=torch.float32, device=H.device)
         _b.vp_ce_forward(H, W, labels, block_v, ignore_index, loss, lse, T_chunk, chunk_index_base, ws)
         ctx.save_for_backward(H, W, labels, lse)
         ctx.cfg = (block_v, ignore_index, T_chunk, chunk_index_base)
-        ctx.ws = ws
         ctx.dW_accum = dW_accum
         return loss
 
@@ -48,15 +45,30 @@ class _VocabProjCE(torch.autograd.Function):
     def backward(ctx, grad_loss):
         H, W, labels, lse = ctx.saved_tensors
         block_v, ignore_index, T_chunk, base = ctx.cfg
-        dH = torch.empty_like(H)
         accum = ctx.dW_accum
-        dW = accum if accum is not None else torch.empty(W.shape, dtype=torch.float32, device=W.device)
+        need_dH = ctx.needs_input_grad[0]
+        need_dW = accum is not None or ctx.needs_input_grad[1]
+        if not (need_dH or need_dW):
+            return (None,) * 8
+        # the workspace holds nothing between calls: it is taken from the caching allocator here, not kept alive
+        # from forward to backward
+        ws = _workspace(T_chunk, H.shape[1], block_v, H.device)
+        dH = torch.empty_like(H) if need_dH else None
+        dW = None
+        if need_dW:
+            dW = accum if accum is not None else torch.empty(W.shape, dtype=torch.float32, device=W.device)
         _b.vp_ce_backward(H, W, labels, lse, grad_loss.to(torch.float32).contiguous(), dH, dW, block_v, ignore_index,
-                          T_chunk, base, accum is not None, ctx.ws)
-        ctx.ws = None
+                          T_chunk, base, accum is not None, ws)
         # with an fp32 accumulation buffer the weight gradient lives there (main-grad style); autograd gets none
-        grad_W = None if accum is not None else dW.to(W.dtype)
+        grad_W = None if (accum is not None or dW is None) else dW.to(W.dtype)
         return dH, grad_W, None, None, None, None, None, None
+
+
+def _workspace(T_chunk: int, d: int, block_v: int, device) -> torch.Tensor:
+    n = _b.vp_ce_workspace_bytes(T_chunk, d, block_v)
+    if n == 0:
+        raise ValueError("unsupported shape: d % 8, block_v % 256 or T_chunk % 128")
+    return torch.empty(n, dtype=torch.uint8, device=device)
 
 
 def vocab_proj_cross_entropy(H: torch.Tensor, W: torch.Tensor, labels: torch.Tensor, block_v: int = 8192,
@@ -88,9 +100,10 @@ class _MaskedMean(torch.autograd.Function):
     @staticmethod
     def backward(ctx, g):
         labels, n_valid = ctx.saved_tensors
-        valid = (labels != ctx.ignore_index) & (labels >= 0) & (labels < ctx.V)
-        inv = torch.where(n_valid > 0, 1.0 / n_valid.clamp(min=1).float(), torch.zeros((), device=g.device))
-        return torch.where(valid, g * inv, torch.zeros((), device=g.device)), None, None, None
+        dloss = torch.empty(labels.numel(), dtype=torch.float32, device=labels.device)
+        _b.vp_ce_mean_loss_grad(labels, ctx.V, ctx.ignore_index, n_valid, g.to(torch.float32).reshape(1).contiguous(),
+                                dloss)
+        return dloss, None, None, None
 
 
 def vocab_proj_cross_entropy_mean(H: torch.Tensor, W: torch.Tensor, labels: torch.Tensor, **kwargs) -> torch.Tensor:

@@ -51,6 +51,8 @@ def load_library() -> ctypes.CDLL:
                                    ctypes.c_int, vp, sz, vp]
     lib.vp_ce_mean_loss.restype = ctypes.c_int
     lib.vp_ce_mean_loss.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
+    lib.vp_ce_mean_loss_grad.restype = ctypes.c_int
+    lib.vp_ce_mean_loss_grad.argtypes = [vp, i64, i64, i32, vp, vp, vp, vp]
     lib.vp_ce_device_status.restype = ctypes.c_int
     lib.vp_ce_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
     lib.vp_ce_status_string.restype = ctypes.c_char_p
@@ -154,7 +156,8 @@ def vp_ce_forward(H, W, labels, block_v: int, ignore_index: int, loss, lse, T_ch
 
 def vp_ce_backward(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index: int, T_chunk: int,
                    chunk_index_base: int, accumulate_dW: bool, workspace, stream=None) -> None:
-    """dH (bf16, overwritten) and dW (fp32, overwritten or accumulated); dloss may be None."""
+    """dH (bf16, overwritten) and dW (fp32, overwritten or accumulated); dloss may be None; one of dH, dW may be
+    None (that gradient is skipped)."""
     import torch
     lib = load_library()
     T, d, V = _shapes(H, W)
@@ -163,10 +166,24 @@ def vp_ce_backward(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index:
             _ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), _ptr(labels, torch.int32, "labels", T),
             _ptr(lse, torch.float32, "lse", T),
             None if dloss is None else _ptr(dloss, torch.float32, "dloss", T),
-            _ptr(dH, torch.bfloat16, "dH", T * d), _ptr(dW, torch.float32, "dW", V * d),
+            None if dH is None else _ptr(dH, torch.bfloat16, "dH", T * d),
+            None if dW is None else _ptr(dW, torch.float32, "dW", V * d),
             T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
             1 if accumulate_dW else 0,
             _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
+
+
+def vp_ce_mean_loss_grad(labels, V: int, ignore_index: int, n_valid, upstream, dloss_out, stream=None) -> None:
+    """dloss_out[n] = upstream / n_valid on valid tokens, 0 elsewhere (upstream may be None = 1)."""
+    import torch
+    lib = load_library()
+    T = labels.numel()
+    with _on_device(labels):
+        _check(lib.vp_ce_mean_loss_grad(
+            _ptr(labels, torch.int32, "labels"), T, int(V), int(ignore_index),
+            _ptr(n_valid, torch.int32, "n_valid", 1),
+            None if upstream is None else _ptr(upstream, torch.float32, "upstream", 1),
+            _ptr(dloss_out, torch.float32, "dloss_out", T), _stream_ptr(stream, labels)))
 
 
 def vp_ce_mean_loss(loss, labels, V: int, ignore_index: int, mean_out, n_valid_out, stream=None) -> None:

@@ -146,16 +146,32 @@ bool make_map_mn3d(CUtensorMap* map, const void* ptr, uint64_t k_rows, uint64_t 
     return r == CUDA_SUCCESS;
 }
 
+// Per-device host-side caches are atomics: concurrent callers may both do the (idempotent) set-up, none reads
+// a half-written value.
 int num_sms() {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (!cached[dev]) {
-        int n = 0;
+    int n = cached[dev].load(std::memory_order_acquire);
+    if (!n) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached[dev] = n;
+        cached[dev].store(n, std::memory_order_release);
     }
-    return cached[dev];
+    return n;
+}
+
+// Raises the dynamic shared-memory limit of `kern` once per device (the attribute is per device and function).
+template <typename K>
+cudaError_t ensure_smem_attr(K kern, int smem_bytes, std::atomic<bool>* done) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (!done[dev].load(std::memory_order_acquire)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        if (e != cudaSuccess) return e;
+        done[dev].store(true, std::memory_order_release);
+    }
+    return cudaSuccess;
 }
 
 template <int BN, bool A_MN, bool B_MN, int EPI>
@@ -163,14 +179,8 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
                         cudaStream_t st) {
     constexpr int SMEM = smem_total<BN, EPI>();
     auto kern = vpce_gemm_kernel<BN, A_MN, B_MN, EPI>;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    }
+    static std::atomic<bool> attr_set[64];
+    if (cudaError_t e = ensure_smem_attr(kern, SMEM, attr_set); e != cudaSuccess) return e;
     const int tiles = p.m_tiles * p.n_tiles;
     if (tiles <= 0 || p.num_kb <= 0) return cudaSuccess;
     const int grid = tiles < num_sms() ? tiles : num_sms();
@@ -197,14 +207,8 @@ cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
                         cudaStream_t st) {
     constexpr int SMEM = pair_smem_total<BN, EPI>();
     auto kern = vpce_gemm_pair_kernel<BN, A_MN, B_MN, EPI, TF32>;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    }
+    static std::atomic<bool> attr_set[64];
+    if (cudaError_t e = ensure_smem_attr(kern, SMEM, attr_set); e != cudaSuccess) return e;
     const int tiles = ((p.m_tiles + 1) / 2) * p.n_tiles;
     if (tiles <= 0 || p.num_kb <= 0) return cudaSuccess;
     const int max_pairs = num_sms() / 2;
@@ -322,9 +326,12 @@ const char* vp_ce_status_string(vpce_status s) {
 
 int64_t vp_ce_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
-                          int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
-                          int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream) {
+// clear_status: whether the call starts by zeroing the device status word (the public entry points do; the
+// backward half of vp_ce_fwd_bwd_host does not, so that what its forward half flagged is still there at the end).
+static vpce_status forward_impl(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
+                                int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
+                                int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream,
+                                bool clear_status) {
     WsLayout L;
     if (T == 0) return VPCE_OK;                                        // empty batch: nothing to compute
     if (!loss || !lse) return VPCE_INVALID_ARG;
@@ -345,8 +352,10 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
         return VPCE_CUDA_ERROR;
     const bool pair_strip = (pair_mask() & 1) != 0;
 
-    vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (clear_status) {
+        vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
     CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
 
     const int64_t P = (V + block_v - 1) / block_v;
@@ -390,10 +399,18 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, i
     return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
 }
 
-vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse, const float* dloss,
-                           void* dH, float* dW, int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
-                           int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW, void* workspace,
-                           size_t workspace_bytes, void* stream) {
+vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
+                          int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
+                          int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream) {
+    return forward_impl(H, W, labels, T, d, V, block_v, ignore_index, loss, lse, T_chunk, chunk_index_base, workspace,
+                        workspace_bytes, stream, true);
+}
+
+static vpce_status backward_impl(const void* H, const void* W, const int32_t* labels, const float* lse,
+                                 const float* dloss, void* dH, float* dW, int64_t T, int64_t d, int64_t V,
+                                 int64_t block_v, int32_t ignore_index, int64_t T_chunk, int64_t chunk_index_base,
+                                 int accumulate_dW, void* workspace, size_t workspace_bytes, void* stream,
+                                 bool clear_status) {
     WsLayout L;
     if (T == 0) {                                                      // empty batch: dW gets no contribution
         if (!accumulate_dW && dW && V > 0 && d > 0 &&
@@ -401,7 +418,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             return VPCE_CUDA_ERROR;
         return VPCE_OK;
     }
-    if (!lse || !dH || !dW) return VPCE_INVALID_ARG;
+    if (!lse || (!dH && !dW)) return VPCE_INVALID_ARG;                 // either gradient may be left out, not both
     vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
     if (s != VPCE_OK) return s;
     if (!aligned16(dH) || !aligned16(dW)) return VPCE_UNSUPPORTED;
@@ -419,8 +436,10 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
         !make_map(&tmG_mn, G, T_chunk, block_v, block_v, 64, BK) || !make_map(&tmH_mn, H, T, d, d, 64, BK))
         return VPCE_CUDA_ERROR;
 
-    vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (clear_status) {
+        vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
     CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
     if (!dloss) {
         vpce_count_valid_kernel<<<1, 1024, 0, st>>>(labels, T, static_cast<int>(V), ignore_index, inv_n, nullptr, status);
@@ -484,14 +503,16 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             ph.b_mn0 = 0; ph.b_k0 = static_cast<int>(v_lo);
             ph.rows_valid = rows; ph.cols_valid = static_cast<int>(d);
             ph.acc = acc; ph.acc_ld = static_cast<int>(d);
-            ph.dH = static_cast<__nv_bfloat16*>(dH) + tok0 * d; ph.out_ld = static_cast<int>(d);
+            ph.dH = dH ? static_cast<__nv_bfloat16*>(dH) + tok0 * d : nullptr; ph.out_ld = static_cast<int>(d);
             ph.first = (i == 0); ph.last = (i == P - 1);
             ph.status = status;
             ph.b_3d = mn3d;
             ph.n_cut = pick_n_cut((ph.m_tiles + 1) / 2, ph.n_tiles, num_sms() / 2);
             apply_tuning(ph, EPI_DH);
             ph.tile_counter = counters.take();
-            if ((pmask & 2) && pair_ok && ph.m_tiles >= 2) {
+            if (!dH) {
+                // input gradient not wanted
+            } else if ((pmask & 2) && pair_ok && ph.m_tiles >= 2) {
                 if (launch_pair<256, false, true, EPI_DH>(tmG_k, tmW_mn2, tmG_k, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
             } else if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) {
                 return VPCE_CUDA_ERROR;
@@ -505,6 +526,7 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             pw.a_mn0 = 0; pw.a_k0 = 0;
             pw.b_mn0 = 0; pw.b_k0 = static_cast<int>(tok0);
             pw.rows_valid = cols; pw.cols_valid = static_cast<int>(d);
+            if (!dW) continue;                                         // weight gradient not wanted
             pw.dW = dW + v_lo * d; pw.out_ld = static_cast<int>(d);
             pw.accumulate = (accumulate_dW != 0) || (c > 0);
             pw.status = status;
@@ -519,14 +541,33 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
             }
         }
     }
-    return VPCE_OK;
+    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
+}
+
+vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse, const float* dloss,
+                           void* dH, float* dW, int64_t T, int64_t d, int64_t V, int64_t block_v, int32_t ignore_index,
+                           int64_t T_chunk, int64_t chunk_index_base, int accumulate_dW, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    return backward_impl(H, W, labels, lse, dloss, dH, dW, T, d, V, block_v, ignore_index, T_chunk, chunk_index_base,
+                         accumulate_dW, workspace, workspace_bytes, stream, true);
 }
 
 vpce_status vp_ce_mean_loss(const float* loss, const int32_t* labels, int64_t T, int64_t V, int32_t ignore_index,
                             float* mean_out, int32_t* n_valid_out, void* stream) {
-    if (!loss || !labels || !mean_out || !n_valid_out || T <= 0 || V <= 0) return VPCE_INVALID_ARG;
+    if (!mean_out || !n_valid_out || T < 0 || V <= 0 || (T > 0 && (!loss || !labels))) return VPCE_INVALID_ARG;
+    // T == 0 (an empty batch) gives mean 0 and n_valid 0, like the empty-batch rule of the other calls
     vpce_mean_loss_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(loss, labels, T, static_cast<int>(V),
                                                                            ignore_index, mean_out, n_valid_out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
+}
+
+vpce_status vp_ce_mean_loss_grad(const int32_t* labels, int64_t T, int64_t V, int32_t ignore_index,
+                                 const int32_t* n_valid, const float* upstream, float* dloss_out, void* stream) {
+    if (!n_valid || T < 0 || V <= 0 || (T > 0 && (!labels || !dloss_out))) return VPCE_INVALID_ARG;
+    if (T == 0) return VPCE_OK;
+    vpce_mean_grad_kernel<<<static_cast<unsigned>((T + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        labels, T, static_cast<int>(V), ignore_index, n_valid, upstream, dloss_out);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
 }
@@ -583,8 +624,9 @@ vpce_status vp_ce_fwd_bwd_host(const void* H_host, const int32_t* labels_host, c
     vpce_status s = vp_ce_forward(H_dev, W, labels_dev, T, d, V, block_v, ignore_index, loss_dev, lse_dev, T_chunk,
                                   chunk_index_base, workspace, workspace_bytes, stream);
     if (s != VPCE_OK) return s;
-    s = vp_ce_backward(H_dev, W, labels_dev, lse_dev, nullptr, dH_dev, dW, T, d, V, block_v, ignore_index, T_chunk,
-                       chunk_index_base, accumulate_dW, workspace, workspace_bytes, stream);
+    // the status word keeps what the forward half flagged: it is cleared once, at the start of the whole pass
+    s = backward_impl(H_dev, W, labels_dev, lse_dev, nullptr, dH_dev, dW, T, d, V, block_v, ignore_index, T_chunk,
+                      chunk_index_base, accumulate_dW, workspace, workspace_bytes, stream, false);
     if (s != VPCE_OK) return s;
     if (cudaMemcpyAsync(loss_host, loss_dev, static_cast<size_t>(T) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return VPCE_CUDA_ERROR;
@@ -653,8 +695,8 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
     if (!make_map(&tmH, H, T, d, d, BK, BM) || !make_map(&tmW, W, V, d, d, BK, BN_VOCAB)) return VPCE_CUDA_ERROR;
     using Cfg = StageCfg<BN_VOCAB>;
     auto kern = vpce_gemm_kernel<BN_VOCAB, false, false, EPI_FOLD>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_TOTAL) != cudaSuccess)
-        return VPCE_CUDA_ERROR;
+    static std::atomic<bool> attr_set[64];
+    if (ensure_smem_attr(kern, Cfg::SMEM_TOTAL, attr_set) != cudaSuccess) return VPCE_CUDA_ERROR;
 
     // The array keeps whatever the previous call left: the status word must start at zero; the
     // running state is initialised by the first merge of every chunk and the partial slots are

@@ -144,6 +144,8 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtens
     const bool row_ok = grow < p.rows_valid;
     int label = row_ok ? p.labels[grow] : p.ignore_index;
     const bool valid = row_ok && label != p.ignore_index && static_cast<unsigned>(label) < static_cast<unsigned>(p.V);
+    // a label outside [0, V) is treated as ignored and flagged (once per row: by the strip's first tile)
+    if (row_ok && !valid && label != p.ignore_index && nt == 0) atomicOr(p.status, VPCE_DEV_LABEL_OUT_OF_RANGE);
     float dl = 0.f, lseL = 0.f;
     if (valid) dl = p.dloss ? p.dloss[grow] : *p.inv_n_valid;
     if (row_ok) lseL = p.lse[grow] * LOG2E;
@@ -197,6 +199,8 @@ __device__ __forceinline__ void epilogue_resid_f32(const GemmParams& p, const CU
     const bool row_ok = grow < p.rows_valid;
     int label = row_ok ? p.labels[grow] : p.ignore_index;
     const bool valid = row_ok && label != p.ignore_index && static_cast<unsigned>(label) < static_cast<unsigned>(p.V);
+    // a label outside [0, V) is treated as ignored and flagged (once per row: by the strip's first tile)
+    if (row_ok && !valid && label != p.ignore_index && nt == 0) atomicOr(p.status, VPCE_DEV_LABEL_OUT_OF_RANGE);
     float dl = 0.f, lseL = 0.f;
     if (valid) dl = p.dloss ? p.dloss[grow] : *p.inv_n_valid;
     if (row_ok) lseL = p.lse[grow] * LOG2E;
@@ -896,6 +900,18 @@ __global__ void vpce_mean_loss_kernel(const float* __restrict__ loss, const int3
         *mean_out = cnts[0] > 0 ? static_cast<float>(sums[0] / cnts[0]) : 0.f;
         *n_valid_out = cnts[0];
     }
+}
+
+// Gradient of the masked mean with respect to the per-token loss: upstream / n_valid on valid tokens, 0 elsewhere.
+__global__ void vpce_mean_grad_kernel(const int32_t* __restrict__ labels, long T, int V, int ignore_index,
+                                      const int* __restrict__ n_valid, const float* __restrict__ upstream,
+                                      float* __restrict__ dloss) {
+    const long i = static_cast<long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= T) return;
+    const int nv = *n_valid;
+    const float g = (upstream ? *upstream : 1.f) * (nv > 0 ? 1.0f / static_cast<float>(nv) : 0.f);
+    const int t = labels[i];
+    dloss[i] = (t != ignore_index && static_cast<unsigned>(t) < static_cast<unsigned>(V)) ? g : 0.f;
 }
 
 __global__ void vpce_clear_status_kernel(int* status) { if (threadIdx.x < 8) status[threadIdx.x] = 0; }

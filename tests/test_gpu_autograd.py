@@ -50,3 +50,39 @@ def test_autograd_per_token_loss_with_fp32_accumulation_buffer():
     assert W.grad is None                                     # the weight gradient went to the fp32 buffer
     assert relF(main_grad.cpu().numpy(), o["dW"]) <= TOL_GRAD
     assert relF(H.grad.float().cpu().numpy(), o["dH"]) <= TOL_GRAD
+
+
+def test_autograd_second_backward_and_frozen_weight():
+    w = custom_workload("ag3", T=256, d=128, V=1500, block_v=512, T_chunk=128, w_std=0.09,
+                        labels="uniform", ignore_frac=0.05, seed=53)
+    b = make_batch(w)
+    o = orc.forward_backward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), b.labels)
+    lab = torch.from_numpy(b.labels).cuda()
+    # a graph that is walked twice (retain_graph): the second backward allocates its own workspace
+    H = to_dev_bf16(b.H_bits).requires_grad_(True)
+    W = to_dev_bf16(b.W_bits).requires_grad_(True)
+    loss = vp.vocab_proj_cross_entropy_mean(H, W, lab, block_v=w.block_v, T_chunk=w.T_chunk)
+    loss.backward(retain_graph=True)
+    g1 = H.grad.clone()
+    H.grad = None
+    loss.backward()
+    assert torch.equal(g1.view(torch.int16), H.grad.view(torch.int16))
+    assert relF(H.grad.float().cpu().numpy(), o["dH"]) <= TOL_GRAD
+    # a frozen projection weight: only the input gradient is computed (the weight-gradient GEMM is skipped)
+    H2 = to_dev_bf16(b.H_bits).requires_grad_(True)
+    W2 = to_dev_bf16(b.W_bits)
+    n0 = vp.vp_ce_launch_count()
+    vp.vocab_proj_cross_entropy_mean(H2, W2, lab, block_v=w.block_v, T_chunk=w.T_chunk).backward()
+    launches_frozen = vp.vp_ce_launch_count() - n0
+    assert relF(H2.grad.float().cpu().numpy(), o["dH"]) <= TOL_GRAD
+    # and the other way round: only the weight gradient
+    H3 = to_dev_bf16(b.H_bits)
+    W3 = to_dev_bf16(b.W_bits).requires_grad_(True)
+    n0 = vp.vp_ce_launch_count()
+    vp.vocab_proj_cross_entropy_mean(H3, W3, lab, block_v=w.block_v, T_chunk=w.T_chunk).backward()
+    assert vp.vp_ce_launch_count() - n0 == launches_frozen
+    assert relF(W3.grad.float().cpu().numpy(), o["dW"]) <= TOL_GRAD
+    meetings = (w.T // w.T_chunk) * w.P
+    n0 = vp.vp_ce_launch_count()
+    vp.vocab_proj_cross_entropy_mean(H, W, lab, block_v=w.block_v, T_chunk=w.T_chunk).backward()
+    assert vp.vp_ce_launch_count() - n0 == launches_frozen + meetings      # one more GEMM per (chunk, shard)

@@ -96,6 +96,12 @@ def test_label_out_of_range_sets_status_and_is_ignored():
     ref = orc.forward_backward(bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits), lab_ok)
     assert np.abs(run.np_loss() - ref["loss"]).max() <= TOL_TOKEN
     assert relF(run.np_dW(), ref["dW"]) <= TOL_GRAD and relF(run.np_dH(), ref["dH"]) <= TOL_GRAD
+    # with an explicit upstream gradient the residual kernel itself must flag it (no label count runs then)
+    dl = orc.default_dloss(lab_ok, IGNORE_INDEX).astype(np.float32)
+    dl[[3, 200]] = 0.25                                     # a non-zero dloss on the bad tokens must still be ignored
+    run.backward(dloss=dl)
+    assert run.bwd_status & 1
+    assert relF(run.np_dW(), ref["dW"]) <= TOL_GRAD and relF(run.np_dH(), ref["dH"]) <= TOL_GRAD
     # a later clean call clears the flag
     run2 = DeviceRun(b.H_bits, b.W_bits, lab_ok, w.block_v, w.T_chunk).forward()
     assert run2.fwd_status == 0
@@ -290,6 +296,23 @@ def test_host_buffer_entry_point_matches_oracle():
     assert relF(dH_h.float().numpy().astype(np.float64), ref["dH"]) <= TOL_GRAD
     assert relF(dW.cpu().numpy().astype(np.float64), ref["dW"]) <= TOL_GRAD
     assert vp.vp_ce_device_status(ws) == 0
+    # the status word read after the call covers BOTH halves: a condition only the forward can raise late in the
+    # pass (here a bad label; the backward flags it too) must not be wiped by the backward's start
+    lh2 = lh.clone().pin_memory()
+    lh2[5] = w.V + 1
+    vp.vp_ce_fwd_bwd_host(Hh, lh2, Wd, loss_h, dH_h, dW, w.block_v, IGNORE_INDEX, w.T_chunk, 0, False,
+                          H_dev, lab_dev, loss_dev, lse_dev, dH_dev, ws)
+    assert vp.vp_ce_device_status(ws) & 1
+    assert float(loss_h[5]) == 0.0 and not dH_h[5].any()
+
+
+def test_mean_loss_of_an_empty_batch_is_zero():
+    mean = torch.full((1,), 7.0, device="cuda")
+    n = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    empty = torch.empty(0, device="cuda")
+    vp.vp_ce_mean_loss(empty, torch.empty(0, dtype=torch.int32, device="cuda"), 1000, IGNORE_INDEX, mean, n)
+    torch.cuda.synchronize()
+    assert float(mean.item()) == 0.0 and int(n.item()) == 0
 
 
 def test_profile_hooks_count_launches_per_kernel_kind():
