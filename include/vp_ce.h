@@ -204,6 +204,29 @@ vpce_status vp_ce_backward_f32(const float* H, const float* W, const int32_t* la
                                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Watchdog of the kernels (no counterpart in the paper).  Every wait inside a kernel (on a copy, on
+ * the tensor cores, on another warp or on the other CTA of a pair) is bounded: when it has lasted
+ * longer than the limit the CTA stops taking work, waits (bounded again) for what it still has in
+ * flight, releases its tensor memory and returns, and VPCE_DEV_WAIT_EXPIRED is set in the status
+ * word; the outputs of that call are then undefined, the context stays usable and the next call
+ * starts clean.  vp_ce_set_wait_limit_ns sets the limit for all later launches of this process
+ * (clamped to [1 ms, 60 s]; ns <= 0 changes nothing) and returns the previous value.  The default
+ * is 2 s.  A kernel that gives up can take up to about twice the limit to return.
+ */
+int64_t vp_ce_set_wait_limit_ns(int64_t ns);
+
+/*
+ * TEST HOOK (no counterpart in the paper): makes one copy of the next launch "get lost" so that
+ * the give-up path above can be exercised without any invalid access.  The next launch of kernel
+ * kind `kernel_kind` (0 forward strip, 1 backward strip, 2 input-gradient GEMM, 3 weight-gradient
+ * GEMM) does not issue the operand copies of k-block `k_block` of the first tile of its work list
+ * in the CTAs named by `cta_ranks` (bit 0: the single CTA or the leader of a CTA pair, bit 1: the
+ * second CTA of a pair); the data simply never arrives.  One-shot: the launch that consumes it
+ * disarms it.  kernel_kind < 0 disarms.  Returns VPCE_INVALID_ARG for values out of range.
+ */
+vpce_status vp_ce_debug_drop_copy(int kernel_kind, int k_block, int cta_ranks);
+
+/*
  * Measurement aid (no counterpart in the paper).  While enabled, every tensor-core kernel
  * launch is bracketed by two CUDA events on the launching stream.  vp_ce_profile_collect
  * waits for the recorded events, adds up the elapsed milliseconds and launch counts per kernel

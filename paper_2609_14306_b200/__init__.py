@@ -17,6 +17,8 @@ from .binding import (  # noqa: F401
     vp_ce_fwd_bwd_host,
     vp_ce_profile_collect,
     vp_ce_profile_enable,
+    vp_ce_set_wait_limit_ns,
+    vp_ce_debug_drop_copy,
     KERNEL_KINDS,
     vp_ce_launch_count,
     vp_ce_mean_loss,

@@ -71,6 +71,10 @@ def load_library() -> ctypes.CDLL:
     lib.vp_ce_backward_f32.restype = ctypes.c_int
     lib.vp_ce_backward_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, i64, i64,
                                        ctypes.c_int, vp, sz, vp]
+    lib.vp_ce_set_wait_limit_ns.restype = i64
+    lib.vp_ce_set_wait_limit_ns.argtypes = [i64]
+    lib.vp_ce_debug_drop_copy.restype = ctypes.c_int
+    lib.vp_ce_debug_drop_copy.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
     lib.vp_ce_profile_enable.restype = None
     lib.vp_ce_profile_enable.argtypes = [ctypes.c_int]
     lib.vp_ce_profile_collect.restype = ctypes.c_int
@@ -234,6 +238,16 @@ def vp_ce_fwd_bwd_host(H_host, labels_host, W, loss_host, dH_host, dW, block_v: 
             _ptr(loss_dev, torch.float32, "loss_dev", T), _ptr(lse_dev, torch.float32, "lse_dev", T),
             _ptr(dH_dev, torch.bfloat16, "dH_dev", T * d),
             _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, W)))
+
+
+def vp_ce_set_wait_limit_ns(ns: int) -> int:
+    """Sets the limit of every wait inside the kernels (ns <= 0: query only); returns the previous limit."""
+    return int(load_library().vp_ce_set_wait_limit_ns(int(ns)))
+
+
+def vp_ce_debug_drop_copy(kernel_kind: int, k_block: int = 0, cta_ranks: int = 1) -> None:
+    """Test hook: the next launch of that kernel kind loses the copies of one k-block (see include/vp_ce.h)."""
+    _check(load_library().vp_ce_debug_drop_copy(int(kernel_kind), int(k_block), int(cta_ranks)))
 
 
 KERNEL_KINDS = ("fwd_strip_fold", "bwd_strip_residual", "dH_gemm", "dW_gemm")

@@ -52,6 +52,26 @@ std::mutex g_prof_mu;
 bool g_prof_on = false;
 std::vector<ProfEntry> g_prof;
 
+// Limit of every wait inside the kernels (vp_ce_set_wait_limit_ns) and the one-shot test hook that makes the next
+// launch of one kernel kind lose a copy (vp_ce_debug_drop_copy): kind in bits 0-7, k-block in bits 8-23, CTA ranks
+// in bits 24-27; -1 = nothing armed.
+std::atomic<unsigned long long> g_wait_limit_ns{kDefaultWaitLimitNs};
+std::atomic<int> g_drop{-1};
+
+// Fills the launch-time fields every GEMM launch shares.
+GemmParams finish_params(const GemmParams& p, int epi) {
+    GemmParams q = p;
+    q.wait_limit_ns = g_wait_limit_ns.load(std::memory_order_relaxed);
+    q.drop_kb = -1;
+    q.drop_ranks = 0;
+    int armed = g_drop.load(std::memory_order_relaxed);
+    if (armed >= 0 && (armed & 0xff) == epi && g_drop.compare_exchange_strong(armed, -1)) {
+        q.drop_kb = (armed >> 8) & 0xffff;
+        q.drop_ranks = (armed >> 24) & 0xf;
+    }
+    return q;
+}
+
 // Tile counters of the dynamic scheduler: one per launch, zeroed in bulk; a call that needs more
 // launches than counters zeroes them again when it wraps (stream order makes that safe).
 constexpr int NUM_TILE_COUNTERS = 1024;
@@ -192,7 +212,7 @@ cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     }
     if (prof && cudaEventCreate(&pe.a) == cudaSuccess && cudaEventCreate(&pe.b) == cudaSuccess) cudaEventRecord(pe.a, st);
     else prof = false;
-    kern<<<grid, NUM_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
+    kern<<<grid, NUM_THREADS, SMEM, st>>>(tmA, tmB, tmC, finish_params(p, EPI));
     if (prof) {
         cudaEventRecord(pe.b, st);
         std::lock_guard<std::mutex> lk(g_prof_mu);
@@ -221,7 +241,7 @@ cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     }
     if (prof && cudaEventCreate(&pe.a) == cudaSuccess && cudaEventCreate(&pe.b) == cudaSuccess) cudaEventRecord(pe.a, st);
     else prof = false;
-    kern<<<grid, NUM_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
+    kern<<<grid, NUM_THREADS, SMEM, st>>>(tmA, tmB, tmC, finish_params(p, EPI));
     if (prof) {
         cudaEventRecord(pe.b, st);
         std::lock_guard<std::mutex> lk(g_prof_mu);
@@ -580,6 +600,24 @@ vpce_status vp_ce_device_status(const void* workspace, int32_t* host_out, void* 
     return cudaStreamSynchronize(st) == cudaSuccess ? VPCE_OK : VPCE_CUDA_ERROR;
 }
 
+int64_t vp_ce_set_wait_limit_ns(int64_t ns) {
+    const unsigned long long prev = g_wait_limit_ns.load(std::memory_order_relaxed);
+    if (ns > 0) {
+        unsigned long long v = static_cast<unsigned long long>(ns);
+        if (v < 1000000ull) v = 1000000ull;                     // at least 1 ms: far longer than any copy is in flight
+        if (v > 60000000000ull) v = 60000000000ull;
+        g_wait_limit_ns.store(v, std::memory_order_relaxed);
+    }
+    return static_cast<int64_t>(prev);
+}
+
+vpce_status vp_ce_debug_drop_copy(int kernel_kind, int k_block, int cta_ranks) {
+    if (kernel_kind < 0) { g_drop.store(-1, std::memory_order_relaxed); return VPCE_OK; }
+    if (kernel_kind > 3 || k_block < 0 || k_block > 0xffff || cta_ranks <= 0 || cta_ranks > 3) return VPCE_INVALID_ARG;
+    g_drop.store(kernel_kind | (k_block << 8) | (cta_ranks << 24), std::memory_order_relaxed);
+    return VPCE_OK;
+}
+
 void vp_ce_profile_enable(int on) {
     std::lock_guard<std::mutex> lk(g_prof_mu);
     g_prof_on = on != 0;
@@ -732,7 +770,7 @@ vpce_status vp_ce_forward_static(const void* H, const void* W, const int32_t* la
             p.tile_counter = counters.take();
             const int tiles = p.m_tiles * p.n_tiles;
             const int grid = tiles < num_sms() ? tiles : num_sms();
-            kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmH, tmW, tmH, p);
+            kern<<<grid, NUM_THREADS, Cfg::SMEM_TOTAL, st>>>(tmH, tmW, tmH, finish_params(p, EPI_FOLD));
             vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
                                                                   rows, i == 0, i == P - 1, labels + tok0, ignore_index,
                                                                   static_cast<int>(V), lse + tok0, loss + tok0, status);

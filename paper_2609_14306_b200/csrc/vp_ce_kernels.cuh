@@ -55,6 +55,12 @@ struct GemmParams {
     int out_ld;
     int* status;
     int* tile_counter;                     // zero before the launch; tiles are taken with atomicAdd
+    unsigned long long wait_limit_ns;      // every wait inside the kernel gives up after this long
+    // Test hook (host-side injection of a lost signal; nothing is accessed out of bounds): the CTA (pair) that takes
+    // list position 0 does not issue the copies of k-block drop_kb of that tile, so the stage's "full" barrier never
+    // completes and the waits run out.  drop_kb < 0: off.  drop_ranks: bit r set = CTA rank r of the pair drops
+    // (bit 0 alone for the single-CTA kernel).
+    int drop_kb, drop_ranks;
 };
 
 template <int BN> struct StageCfg {
@@ -406,7 +412,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             };
             while (ok) {
-                if (!mbar_wait(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(sempty_bar(ss), sphase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                 int tile = atomicAdd(p.tile_counter, 1);
                 if (tile >= total_tiles) tile = -1;
                 sched_slot[ss] = tile;
@@ -416,10 +422,11 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 int mt, nt;
                 decode_tile(p, tile, mt, nt);
                 for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-                    issue(mt, nt, kb, sa, sa + Cfg::A_BYTES, full_bar(stage));
+                    const bool drop = tile == 0 && kb == p.drop_kb && (p.drop_ranks & 1);   // test hook: a lost copy
+                    if (!drop) issue(mt, nt, kb, sa, sa + Cfg::A_BYTES, full_bar(stage));
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -431,7 +438,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (long i = 0; i < back; ++i) {
                     if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
                     unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < p.wait_limit_ns) {}
                 }
             }
         }
@@ -441,7 +448,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int stage = 0; uint32_t phase = 0; bool ok = true;
             int ss = 0; uint32_t sphase = 0;
             for (int it = 0; ok; ++it) {
-                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                 const int tile = sched_slot[ss];
                 mbar_arrive(sempty_bar(ss));
                 if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
@@ -451,11 +458,11 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const uint32_t idesc = make_idesc(tile_n(nt), A_MN, B_MN, BM);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
-                if (!mbar_wait(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar(ab), aphase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
                     const uint32_t sb = sa + Cfg::A_BYTES;
@@ -476,7 +483,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ok || *abort_flag) {
                 umma_commit(drain_bar);                                 // wait for MMAs still in flight
                 unsigned long long t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < p.wait_limit_ns) {}
             }
         }
     } else {
@@ -488,7 +495,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int it = 0; ok; ++it) {
             int tile = -2;
             if (lane == 0) {
-                if (mbar_wait(sfull_bar(ss), sphase, abort_flag)) {
+                if (mbar_wait(sfull_bar(ss), sphase, abort_flag, p.wait_limit_ns)) {
                     tile = sched_slot[ss];
                     mbar_arrive(sempty_bar(ss));
                 }
@@ -500,7 +507,7 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             decode_tile(p, tile, mt, nt);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
             tc_fence_after();
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
@@ -670,7 +677,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             bool exhausted = false;
             auto publish = [&]() -> int {
                 if (exhausted) return -1;
-                if (!mbar_wait_cluster(sempty_bar(ss), sphase ^ 1u, abort_flag)) { ok = false; return -1; }
+                if (!mbar_wait_cluster(sempty_bar(ss), sphase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; return -1; }
                 int t = atomicAdd(p.tile_counter, 1);
                 if (t >= list_len) { t = -1; exhausted = true; }
                 sched_slot[ss] = t;
@@ -688,7 +695,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (tile >= 0) ahead = publish();
                     if (!ok) break;
                 } else {
-                    if (!mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     tile = sched_slot[ss];
                     sched_ack(ss);
                     if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
@@ -700,15 +707,18 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
                 const int bn0 = ncol0 + static_cast<int>(rank) * (width / 2);   // this CTA's half of the B tile
                 for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
                     const uint32_t bar = mapa_shared(full_bar(stage), 0);    // the leader's barrier
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
                     const uint32_t sb = sa + Cfg::A_BYTES;
-                    if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BKE, (p.a_mn0 + mt * BM) >> CSH, pol_a);
-                    else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BKE, p.a_mn0 + mt * BM, pol_a);
-                    if (B_MN) tma2_load_3d(sb, &tmB, bar, 0, p.b_k0 + kb * BKE, (p.b_mn0 + bn0) >> CSH, pol_b);
-                    else tma2_load_2d(sb, &tmB, bar, p.b_k0 + kb * BKE, p.b_mn0 + bn0, pol_b);
+                    const bool drop = tile == 0 && kb == p.drop_kb && ((p.drop_ranks >> rank) & 1);   // test hook
+                    if (!drop) {
+                        if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BKE, (p.a_mn0 + mt * BM) >> CSH, pol_a);
+                        else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BKE, p.a_mn0 + mt * BM, pol_a);
+                        if (B_MN) tma2_load_3d(sb, &tmB, bar, 0, p.b_k0 + kb * BKE, (p.b_mn0 + bn0) >> CSH, pol_b);
+                        else tma2_load_2d(sb, &tmB, bar, p.b_k0 + kb * BKE, p.b_mn0 + bn0, pol_b);
+                    }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -720,7 +730,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 for (long i = 0; i < back; ++i) {
                     if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
                     unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(full_bar(s), ph) && globaltimer_ns() - t0 < p.wait_limit_ns) {}
                 }
             }
         }
@@ -730,7 +740,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int stage = 0; uint32_t phase = 0; bool ok = true;
             int ss = 0; uint32_t sphase = 0;
             for (int it = 0; ok;) {
-                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(sfull_bar(ss), sphase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                 const int tile = sched_slot[ss];
                 sched_ack(ss);
                 if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
@@ -741,11 +751,11 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM, TF32 ? 2u : 1u);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
-                if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
                     const uint32_t sb = sa + Cfg::A_BYTES;
@@ -771,7 +781,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (!ok || *abort_flag) {
                 umma2_commit_local(drain_bar);
                 unsigned long long t0 = globaltimer_ns();
-                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(drain_bar, 0) && globaltimer_ns() - t0 < p.wait_limit_ns) {}
             }
         }
     } else {
@@ -783,7 +793,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         for (int it = 0; ok;) {
             int tile = -2;
             if (lane == 0) {
-                if (mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag)) {
+                if (mbar_wait_cluster(sfull_bar(ss), sphase, abort_flag, p.wait_limit_ns)) {
                     tile = sched_slot[ss];
                     sched_ack(ss);
                 }
@@ -797,7 +807,7 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             const int mt = 2 * pmt + static_cast<int>(rank);
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(tfull_bar(ab), aphase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
             tc_fence_after();
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);

@@ -52,3 +52,19 @@ def test_status_strings():
         assert vp.vp_ce_status_string(c) not in ("ok", "unknown status")
     assert vp.vp_ce_status_string(99) == "unknown status"
     assert vp.vp_ce_launch_count() >= 0
+
+
+def test_wait_limit_and_test_hook_arguments():
+    # pure host state: no kernel is launched
+    prev = vp.vp_ce_set_wait_limit_ns(0)                      # query only
+    assert prev == 2_000_000_000
+    assert vp.vp_ce_set_wait_limit_ns(5) == prev              # clamped up to 1 ms ...
+    assert vp.vp_ce_set_wait_limit_ns(10**12) == 1_000_000    # ... and down to 60 s
+    assert vp.vp_ce_set_wait_limit_ns(prev) == 60_000_000_000
+    assert vp.vp_ce_set_wait_limit_ns(-1) == prev
+    import pytest
+    for bad in [(4, 0, 1), (0, -1, 1), (0, 0, 0), (0, 0, 4), (0, 70000, 1)]:
+        with pytest.raises(vp.VpceError):
+            vp.vp_ce_debug_drop_copy(*bad)
+    vp.vp_ce_debug_drop_copy(2, 3, 3)
+    vp.vp_ce_debug_drop_copy(-1)                              # disarm
