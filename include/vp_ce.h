@@ -94,6 +94,45 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Single meetings, for a ring driver that runs Algorithm 3 ACROSS devices (each rank holds its own batch
+ * X_r [N, d] with targets t_r and owns shard W_r, the rows [v_lo, v_lo + shard_rows) of the weight; either
+ * the shard or the batch travels around the ring, section 3.2 "Which tensor travels").  One call = one
+ * meeting of a batch with a shard; everything it touches is in this device's memory.
+ *
+ * vp_ce_meeting_forward: forms the strip X W_shard^T and folds it into the batch's running state (Eq. 2;
+ * Algorithm 3, Fold).  state is the caller's DEVICE array [3][N] fp32 = (m, z, y_t): it stays on the rank in
+ * the move-weights schedule and travels with (X, t) in the move-activations schedule.  first != 0: the
+ * state starts from (-inf, 0, 0) (its previous contents are ignored) and the status word is cleared;
+ * last != 0: lse[n] = m + log z and loss[n] = lse[n] - y_t (0 if ignored) are written as well.
+ * shard_rows and N need not be multiples of the tile shapes.
+ *
+ * vp_ce_meeting_backward: the backward meeting (Appendix C), in up to three phases selected by `phases`
+ * so that a ring driver can wait for a travelling accumulator between them:
+ *   VPCE_PHASE_RESIDUAL     recompute the strip, residual G = dloss (exp(Y - lse) - onehot) -> workspace
+ *   VPCE_PHASE_INPUT_GRAD   dX_acc (+)= G W_shard   fp32 [N, d]; first != 0 overwrites; last != 0 writes the
+ *                           final bf16 dX [N, d] instead of the accumulator (dX_acc is read unless first)
+ *   VPCE_PHASE_WEIGHT_GRAD  dW_shard (+)= G^T X     fp32 [shard_rows, d]; accumulate_dW == 0 overwrites
+ * The gradient of the tensor that travels goes with it: dX_acc in the move-activations schedule, dW_shard
+ * in the move-weights schedule.  Phases of one meeting must use the same workspace, in this order, with
+ * nothing else using it in between.  dloss is required (the ring driver knows the global token count).
+ *
+ * vp_ce_meeting_workspace_bytes(N, d, shard_rows): bytes both calls need (O(N * shard_rows), Eq. 1).
+ */
+#define VPCE_PHASE_RESIDUAL    1
+#define VPCE_PHASE_INPUT_GRAD  2
+#define VPCE_PHASE_WEIGHT_GRAD 4
+size_t vp_ce_meeting_workspace_bytes(int64_t N, int64_t d, int64_t shard_rows);
+vpce_status vp_ce_meeting_forward(const void* X, const void* W_shard, const int32_t* targets,
+                                  int64_t N, int64_t d, int64_t shard_rows, int64_t v_lo, int64_t V,
+                                  int32_t ignore_index, float* state, int first, int last,
+                                  float* loss, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+vpce_status vp_ce_meeting_backward(const void* X, const void* W_shard, const int32_t* targets, const float* lse,
+                                   const float* dloss, int64_t N, int64_t d, int64_t shard_rows, int64_t v_lo,
+                                   int64_t V, int32_t ignore_index, int phases, float* dX_acc, int first, int last,
+                                   void* dX, float* dW_shard, int accumulate_dW,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Masked mean of the per-token loss (not part of the paper's operator, which outputs
  * per-token values; this is the reduction the benchmark's metric is stated on).
  * mean_out[0] = sum of loss over valid tokens / n_valid (0 when n_valid == 0);

@@ -22,6 +22,12 @@ from .binding import (  # noqa: F401
     KERNEL_KINDS,
     vp_ce_launch_count,
     vp_ce_mean_loss,
+    vp_ce_meeting_backward,
+    vp_ce_meeting_forward,
+    vp_ce_meeting_workspace_bytes,
+    PHASE_RESIDUAL,
+    PHASE_INPUT_GRAD,
+    PHASE_WEIGHT_GRAD,
     vp_ce_mean_loss_grad,
     vp_ce_status_string,
     vp_ce_workspace_bytes,

@@ -51,6 +51,14 @@ def load_library() -> ctypes.CDLL:
                                    ctypes.c_int, vp, sz, vp]
     lib.vp_ce_mean_loss.restype = ctypes.c_int
     lib.vp_ce_mean_loss.argtypes = [vp, vp, i64, i64, i32, vp, vp, vp]
+    lib.vp_ce_meeting_workspace_bytes.restype = sz
+    lib.vp_ce_meeting_workspace_bytes.argtypes = [i64, i64, i64]
+    lib.vp_ce_meeting_forward.restype = ctypes.c_int
+    lib.vp_ce_meeting_forward.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp, ctypes.c_int, ctypes.c_int,
+                                          vp, vp, vp, sz, vp]
+    lib.vp_ce_meeting_backward.restype = ctypes.c_int
+    lib.vp_ce_meeting_backward.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i32, ctypes.c_int, vp,
+                                           ctypes.c_int, ctypes.c_int, vp, vp, ctypes.c_int, vp, sz, vp]
     lib.vp_ce_mean_loss_grad.restype = ctypes.c_int
     lib.vp_ce_mean_loss_grad.argtypes = [vp, i64, i64, i32, vp, vp, vp, vp]
     lib.vp_ce_device_status.restype = ctypes.c_int
@@ -175,6 +183,50 @@ def vp_ce_backward(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_index:
             T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
             1 if accumulate_dW else 0,
             _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
+
+
+PHASE_RESIDUAL, PHASE_INPUT_GRAD, PHASE_WEIGHT_GRAD = 1, 2, 4
+
+
+def vp_ce_meeting_workspace_bytes(N: int, d: int, shard_rows: int) -> int:
+    return int(load_library().vp_ce_meeting_workspace_bytes(int(N), int(d), int(shard_rows)))
+
+
+def vp_ce_meeting_forward(X, W_shard, targets, v_lo: int, V: int, ignore_index: int, state, first: bool, last: bool,
+                          loss, lse, workspace, stream=None) -> None:
+    """One forward meeting of batch X [N, d] with shard W_shard (vocabulary ids v_lo ...): folds the strip into
+    state [3, N] = (m, z, y_t); with last=True also writes lse and loss."""
+    import torch
+    lib = load_library()
+    N, d, S = _shapes(X, W_shard)
+    with _on_device(X):
+        _check(lib.vp_ce_meeting_forward(
+            _ptr(X, torch.bfloat16, "X"), _ptr(W_shard, torch.bfloat16, "W_shard"),
+            _ptr(targets, torch.int32, "targets", N), N, d, S, int(v_lo), int(V), int(ignore_index),
+            _ptr(state, torch.float32, "state", 3 * N), 1 if first else 0, 1 if last else 0,
+            None if loss is None else _ptr(loss, torch.float32, "loss", N),
+            None if lse is None else _ptr(lse, torch.float32, "lse", N),
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, X)))
+
+
+def vp_ce_meeting_backward(X, W_shard, targets, lse, dloss, v_lo: int, V: int, ignore_index: int, phases: int,
+                           dX_acc, first: bool, last: bool, dX, dW_shard, accumulate_dW: bool, workspace,
+                           stream=None) -> None:
+    """One backward meeting (phases: bit mask of PHASE_*); see include/vp_ce.h."""
+    import torch
+    lib = load_library()
+    N, d, S = _shapes(X, W_shard)
+    with _on_device(X):
+        _check(lib.vp_ce_meeting_backward(
+            _ptr(X, torch.bfloat16, "X"), _ptr(W_shard, torch.bfloat16, "W_shard"),
+            _ptr(targets, torch.int32, "targets", N), _ptr(lse, torch.float32, "lse", N),
+            _ptr(dloss, torch.float32, "dloss", N), N, d, S, int(v_lo), int(V), int(ignore_index), int(phases),
+            None if dX_acc is None else _ptr(dX_acc, torch.float32, "dX_acc", N * d),
+            1 if first else 0, 1 if last else 0,
+            None if dX is None else _ptr(dX, torch.bfloat16, "dX", N * d),
+            None if dW_shard is None else _ptr(dW_shard, torch.float32, "dW_shard", S * d),
+            1 if accumulate_dW else 0,
+            _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, X)))
 
 
 def vp_ce_mean_loss_grad(labels, V: int, ignore_index: int, n_valid, upstream, dloss_out, stream=None) -> None:

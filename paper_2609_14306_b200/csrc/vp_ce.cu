@@ -321,6 +321,279 @@ vpce_status check_common(const void* H, const void* W, const int32_t* labels, in
     return VPCE_OK;
 }
 
+// ------------------------------------------------------------------------------------ one meeting
+// A "meeting" is what Algorithm 3 does when one token batch X (rows) is co-located with one vocabulary shard
+// W_q (cols rows of the weight): forward = form the strip X W_q^T and fold it into the batch's running state;
+// backward = recompute the strip, form the residual and contract it into the two gradients.  vp_ce_forward /
+// vp_ce_backward loop over (chunk, shard) meetings on one device; vp_ce_meeting_* expose a single meeting to a
+// ring driver that moves the shard or the batch between devices.
+
+// Tensor maps and workspace pointers of the forward meetings of one call.
+struct FoldCtx {
+    CUtensorMap tmX, tmW, tmW_half;
+    int* status; float *sm, *sz, *ylab, *pm, *pz;
+    int part_ld, num_kb, ignore_index, V;
+    int64_t d;
+    bool pair_strip;
+};
+
+bool make_fold_ctx(FoldCtx* c, const void* X, int64_t x_rows, const void* W, int64_t w_rows, int64_t d) {
+    c->d = d;
+    c->num_kb = static_cast<int>((d + BK - 1) / BK);
+    c->pair_strip = (pair_mask() & 1) != 0;
+    return make_map(&c->tmX, X, x_rows, d, d, BK, BM) && make_map(&c->tmW, W, w_rows, d, d, BK, BN_VOCAB) &&
+           make_map(&c->tmW_half, W, w_rows, d, d, BK, BN_VOCAB / 2);
+}
+
+// Forward meeting: rows [x_row0, x_row0 + rows) of the X map meet rows [w_row0, w_row0 + cols) of the W map, which
+// are vocabulary ids [v_lo, v_lo + cols).  labels / lse / loss point at the batch's first token.  first: the state
+// starts from (-inf, 0, 0); last: lse and loss are emitted (Algorithm 3, output line).
+cudaError_t fold_meeting(const FoldCtx& c, int x_row0, int rows, int w_row0, int cols, int v_lo, const int32_t* labels,
+                         bool first, bool last, float* lse, float* loss, CounterPool& counters, cudaStream_t st) {
+    GemmParams p{};
+    p.m_tiles = (rows + BM - 1) / BM;
+    p.n_tiles = (cols + BN_VOCAB - 1) / BN_VOCAB;
+    p.num_kb = c.num_kb;
+    p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * c.d);
+    p.a_mn0 = x_row0; p.a_k0 = 0;
+    p.b_mn0 = w_row0; p.b_k0 = 0;
+    p.rows_valid = rows; p.cols_valid = cols;
+    p.v_lo = v_lo;
+    p.labels = labels;
+    p.ignore_index = c.ignore_index; p.V = c.V;
+    p.pm = c.pm; p.pz = c.pz; p.ylab = c.ylab; p.part_ld = c.part_ld;
+    p.status = c.status;
+    apply_tuning(p, EPI_FOLD);
+    p.tile_counter = counters.take();
+    cudaError_t e;
+    if (c.pair_strip && p.m_tiles >= 2) e = launch_pair<BN_VOCAB, false, false, EPI_FOLD>(c.tmX, c.tmW_half, c.tmX, p, st);
+    else e = launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(c.tmX, c.tmW, c.tmX, p, st);
+    if (e != cudaSuccess) return e;
+    vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(c.pm, c.pz, c.part_ld, p.n_tiles, c.sm, c.sz, c.ylab, rows, first,
+                                                          last, labels, c.ignore_index, c.V, lse, loss, c.status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+// Tensor maps and workspace pointers of the backward meetings of one call.
+struct GradCtx {
+    CUtensorMap tmX_k, tmW_k, tmW_khalf, tmG_st, tmG_k, tmW_mn, tmG_mn, tmX_mn, tmW_mn2, tmX_mn2;
+    int* status; float* inv_n; __nv_bfloat16* G;
+    int g_rows, g_ld;                       // rows and row pitch (elements) of the residual strip in the workspace
+    int bn, pmask, ignore_index, V;
+    int64_t d;
+    bool pair_ok, mn3d;
+};
+
+bool make_grad_ctx(GradCtx* c, const void* X, int64_t x_rows, const void* W, int64_t w_rows, int64_t d,
+                   __nv_bfloat16* G, int64_t g_rows, int64_t g_ld) {
+    c->d = d; c->G = G; c->g_rows = static_cast<int>(g_rows); c->g_ld = static_cast<int>(g_ld);
+    c->bn = pick_bn(d);
+    c->pmask = pair_mask();
+    c->pair_ok = (c->bn == 256) && (d % 64 == 0);
+    c->mn3d = (d % 64 == 0);             // one-instruction fetch of MN-major operands when the contiguous extent allows
+    if (!make_map(&c->tmG_st, G, g_rows, g_ld, g_ld, 64, 32) ||
+        !make_map(&c->tmX_k, X, x_rows, d, d, BK, BM) || !make_map(&c->tmW_k, W, w_rows, d, d, BK, BN_VOCAB) ||
+        !make_map(&c->tmW_khalf, W, w_rows, d, d, BK, BN_VOCAB / 2) ||
+        !make_map(&c->tmG_k, G, g_rows, g_ld, g_ld, BK, BM) || !make_map(&c->tmW_mn, W, w_rows, d, d, 64, BK) ||
+        !make_map(&c->tmG_mn, G, g_rows, g_ld, g_ld, 64, BK) || !make_map(&c->tmX_mn, X, x_rows, d, d, 64, BK))
+        return false;
+    // CTA-pair variants: half-width B boxes
+    if (c->pair_ok && (!make_map_mn3d(&c->tmW_mn2, W, w_rows, d, d, 2) || !make_map_mn3d(&c->tmX_mn2, X, x_rows, d, d, 2)))
+        return false;
+    if (c->mn3d && (!make_map_mn3d(&c->tmW_mn, W, w_rows, d, d, c->bn / 64) ||
+                    !make_map_mn3d(&c->tmX_mn, X, x_rows, d, d, c->bn / 64) ||
+                    !make_map_mn3d(&c->tmG_mn, G, g_rows, g_ld, g_ld, BM / 64)))
+        return false;
+    return true;
+}
+
+enum { PHASE_RESIDUAL = VPCE_PHASE_RESIDUAL, PHASE_INPUT_GRAD = VPCE_PHASE_INPUT_GRAD,
+       PHASE_WEIGHT_GRAD = VPCE_PHASE_WEIGHT_GRAD };
+
+// Backward meeting, in up to three phases (a ring driver may wait for a travelling accumulator between them):
+//   residual     recompute the strip, G = dloss (exp(Y - lse) - onehot) as bf16 into the workspace
+//   input grad   acc (+)= G W_q   (fp32 [rows, d], pitch d; first: overwrite; last: write bf16 dX instead)
+//   weight grad  dW_q (+)= G^T X  (fp32 [cols, d])
+// labels / lse / dloss / acc / dX point at the batch's first token, dW_q at the shard's first row.
+cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int w_row0, int cols, int v_lo,
+                         const int32_t* labels, const float* lse, const float* dloss, bool first, bool last, float* acc,
+                         __nv_bfloat16* dX, float* dW_q, bool accumulate_dW, CounterPool& counters, cudaStream_t st) {
+    const int strip_tiles_n = (cols + BN_VOCAB - 1) / BN_VOCAB;
+    const int m_tiles = (rows + BM - 1) / BM;
+    const int d = static_cast<int>(c.d);
+    cudaError_t e = cudaSuccess;
+    if (phases & PHASE_RESIDUAL) {
+        GemmParams p{};
+        p.m_tiles = m_tiles;
+        p.n_tiles = strip_tiles_n;
+        p.num_kb = (d + BK - 1) / BK;
+        p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * d);
+        p.a_mn0 = x_row0; p.b_mn0 = w_row0;
+        p.rows_valid = rows; p.cols_valid = cols;
+        p.v_lo = v_lo;
+        p.labels = labels; p.lse = lse; p.dloss = dloss;
+        p.inv_n_valid = c.inv_n; p.ignore_index = c.ignore_index; p.V = c.V;
+        p.G = c.G; p.g_ld = c.g_ld; p.g_rows = c.g_rows;
+        p.status = c.status;
+        apply_tuning(p, EPI_RESID);
+        p.tile_counter = counters.take();
+        if ((c.pmask & 1) && p.m_tiles >= 2) e = launch_pair<BN_VOCAB, false, false, EPI_RESID>(c.tmX_k, c.tmW_khalf, c.tmG_st, p, st);
+        else e = launch_gemm<BN_VOCAB, false, false, EPI_RESID>(c.tmX_k, c.tmW_k, c.tmG_st, p, st);
+        if (e != cudaSuccess) return e;
+    }
+    const int k_cols = strip_tiles_n * BN_VOCAB;               // columns of G written by the residual phase
+    const int m_rows = m_tiles * BM;                           // rows of G written by the residual phase
+    const int grad_n_tiles = (d + c.bn - 1) / c.bn;
+    if (phases & PHASE_INPUT_GRAD) {
+        // dX += G W_q : M = tokens, N = d, K = shard vocabulary
+        GemmParams ph{};
+        ph.m_tiles = m_tiles;
+        ph.n_tiles = grad_n_tiles;
+        ph.num_kb = k_cols / BK;
+        ph.group_n = pick_group_n(ph.n_tiles, 2.0 * k_cols * d);
+        ph.a_mn0 = 0; ph.a_k0 = 0;
+        ph.b_mn0 = 0; ph.b_k0 = w_row0;
+        ph.rows_valid = rows; ph.cols_valid = d;
+        ph.acc = acc; ph.acc_ld = d;
+        ph.dH = dX; ph.out_ld = d;
+        ph.first = first; ph.last = last;
+        ph.status = c.status;
+        ph.b_3d = c.mn3d;
+        ph.n_cut = pick_n_cut((ph.m_tiles + 1) / 2, ph.n_tiles, num_sms() / 2);
+        apply_tuning(ph, EPI_DH);
+        ph.tile_counter = counters.take();
+        if ((c.pmask & 2) && c.pair_ok && ph.m_tiles >= 2) e = launch_pair<256, false, true, EPI_DH>(c.tmG_k, c.tmW_mn2, c.tmG_k, ph, st);
+        else e = launch_grad<false, true, EPI_DH>(c.bn, c.tmG_k, c.tmW_mn, ph, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (phases & PHASE_WEIGHT_GRAD) {
+        // dW_q += G^T X : M = shard vocabulary, N = d, K = batch tokens
+        GemmParams pw{};
+        pw.m_tiles = (cols + BM - 1) / BM;
+        pw.n_tiles = grad_n_tiles;
+        pw.num_kb = m_rows / BK;
+        pw.group_n = pick_group_n(pw.n_tiles, 2.0 * m_rows * d);
+        pw.a_mn0 = 0; pw.a_k0 = 0;
+        pw.b_mn0 = 0; pw.b_k0 = x_row0;
+        pw.rows_valid = cols; pw.cols_valid = d;
+        pw.dW = dW_q; pw.out_ld = d;
+        pw.accumulate = accumulate_dW;
+        pw.status = c.status;
+        pw.a_3d = c.mn3d; pw.b_3d = c.mn3d;
+        pw.n_cut = pick_n_cut((pw.m_tiles + 1) / 2, pw.n_tiles, num_sms() / 2);
+        apply_tuning(pw, EPI_DW);
+        pw.tile_counter = counters.take();
+        if ((c.pmask & 4) && c.pair_ok && pw.m_tiles >= 2) e = launch_pair<256, true, true, EPI_DW>(c.tmG_mn, c.tmX_mn2, c.tmG_mn, pw, st);
+        else e = launch_grad<true, true, EPI_DW>(c.bn, c.tmG_mn, c.tmX_mn, pw, st);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// clear_status: whether the call starts by zeroing the device status word (the public entry points do; the
+// backward half of vp_ce_fwd_bwd_host does not, so that what its forward half flagged is still there at the end).
+vpce_status forward_impl(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
+                         int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
+                         int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream,
+                         bool clear_status) {
+    WsLayout L;
+    if (T == 0) return VPCE_OK;                                        // empty batch: nothing to compute
+    if (!loss || !lse) return VPCE_INVALID_ARG;
+    vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
+    if (s != VPCE_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    FoldCtx c;
+    if (!make_fold_ctx(&c, H, T, W, V, d)) return VPCE_CUDA_ERROR;
+    c.status = reinterpret_cast<int*>(ws + L.status);
+    c.sm = reinterpret_cast<float*>(ws + L.sm);
+    c.sz = reinterpret_cast<float*>(ws + L.sz);
+    c.ylab = reinterpret_cast<float*>(ws + L.ylab);
+    c.pm = reinterpret_cast<float*>(ws + L.pm);
+    c.pz = reinterpret_cast<float*>(ws + L.pz);
+    c.part_ld = static_cast<int>(T_chunk);
+    c.ignore_index = ignore_index; c.V = static_cast<int>(V);
+
+    if (clear_status) {
+        vpce_clear_status_kernel<<<1, 32, 0, st>>>(c.status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
+
+    const int64_t P = (V + block_v - 1) / block_v;
+    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
+    for (int64_t ch = 0; ch < n_chunks; ++ch) {
+        const int64_t tok0 = ch * T_chunk;
+        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
+        const int64_t cg = chunk_index_base + ch;
+        for (int64_t i = 0; i < P; ++i) {
+            const int64_t q = ((cg - i) % P + P) % P;                  // Algorithm 3: q = (r - i) mod P
+            const int64_t v_lo = q * block_v;
+            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
+            if (fold_meeting(c, static_cast<int>(tok0), rows, static_cast<int>(v_lo), cols, static_cast<int>(v_lo),
+                             labels + tok0, i == 0, i == P - 1, lse + tok0, loss + tok0, counters, st) != cudaSuccess)
+                return VPCE_CUDA_ERROR;
+        }
+    }
+    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
+}
+
+vpce_status backward_impl(const void* H, const void* W, const int32_t* labels, const float* lse,
+                          const float* dloss, void* dH, float* dW, int64_t T, int64_t d, int64_t V,
+                          int64_t block_v, int32_t ignore_index, int64_t T_chunk, int64_t chunk_index_base,
+                          int accumulate_dW, void* workspace, size_t workspace_bytes, void* stream,
+                          bool clear_status) {
+    WsLayout L;
+    if (T == 0) {                                                      // empty batch: dW gets no contribution
+        if (!accumulate_dW && dW && V > 0 && d > 0 &&
+            cudaMemsetAsync(dW, 0, static_cast<size_t>(V) * d * 4, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return VPCE_CUDA_ERROR;
+        return VPCE_OK;
+    }
+    if (!lse || (!dH && !dW)) return VPCE_INVALID_ARG;                 // either gradient may be left out, not both
+    vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
+    if (s != VPCE_OK) return s;
+    if (!aligned16(dH) || !aligned16(dW)) return VPCE_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    GradCtx c;
+    if (!make_grad_ctx(&c, H, T, W, V, d, reinterpret_cast<__nv_bfloat16*>(ws + L.G), T_chunk, block_v)) return VPCE_CUDA_ERROR;
+    c.status = reinterpret_cast<int*>(ws + L.status);
+    c.inv_n = reinterpret_cast<float*>(ws + L.scalars);
+    c.ignore_index = ignore_index; c.V = static_cast<int>(V);
+    float* acc = reinterpret_cast<float*>(ws + L.acc);
+
+    if (clear_status) {
+        vpce_clear_status_kernel<<<1, 32, 0, st>>>(c.status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
+    if (!dloss) {
+        vpce_count_valid_kernel<<<1, 1024, 0, st>>>(labels, T, static_cast<int>(V), ignore_index, c.inv_n, nullptr, c.status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    const int phases = PHASE_RESIDUAL | (dH ? PHASE_INPUT_GRAD : 0) | (dW ? PHASE_WEIGHT_GRAD : 0);
+    const int64_t P = (V + block_v - 1) / block_v;
+    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
+    for (int64_t ch = 0; ch < n_chunks; ++ch) {
+        const int64_t tok0 = ch * T_chunk;
+        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
+        const int64_t cg = chunk_index_base + ch;
+        for (int64_t i = 0; i < P; ++i) {
+            const int64_t q = ((cg - i) % P + P) % P;
+            const int64_t v_lo = q * block_v;
+            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
+            if (grad_meeting(c, phases, static_cast<int>(tok0), rows, static_cast<int>(v_lo), cols, static_cast<int>(v_lo),
+                             labels + tok0, lse + tok0, dloss ? dloss + tok0 : nullptr, i == 0, i == P - 1, acc,
+                             dH ? static_cast<__nv_bfloat16*>(dH) + tok0 * d : nullptr, dW ? dW + v_lo * d : nullptr,
+                             (accumulate_dW != 0) || (ch > 0), counters, st) != cudaSuccess)
+                return VPCE_CUDA_ERROR;
+        }
+    }
+    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------ C ABI
@@ -346,222 +619,11 @@ const char* vp_ce_status_string(vpce_status s) {
 
 int64_t vp_ce_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-// clear_status: whether the call starts by zeroing the device status word (the public entry points do; the
-// backward half of vp_ce_fwd_bwd_host does not, so that what its forward half flagged is still there at the end).
-static vpce_status forward_impl(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
-                                int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
-                                int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream,
-                                bool clear_status) {
-    WsLayout L;
-    if (T == 0) return VPCE_OK;                                        // empty batch: nothing to compute
-    if (!loss || !lse) return VPCE_INVALID_ARG;
-    vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
-    if (s != VPCE_OK) return s;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    int* status = reinterpret_cast<int*>(ws + L.status);
-    float* sm = reinterpret_cast<float*>(ws + L.sm);
-    float* sz = reinterpret_cast<float*>(ws + L.sz);
-    float* ylab = reinterpret_cast<float*>(ws + L.ylab);
-    float* pm = reinterpret_cast<float*>(ws + L.pm);
-    float* pz = reinterpret_cast<float*>(ws + L.pz);
-
-    CUtensorMap tmH, tmW, tmW_half;
-    if (!make_map(&tmH, H, T, d, d, BK, BM) || !make_map(&tmW, W, V, d, d, BK, BN_VOCAB) ||
-        !make_map(&tmW_half, W, V, d, d, BK, BN_VOCAB / 2))
-        return VPCE_CUDA_ERROR;
-    const bool pair_strip = (pair_mask() & 1) != 0;
-
-    if (clear_status) {
-        vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-    }
-    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
-
-    const int64_t P = (V + block_v - 1) / block_v;
-    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
-    const int num_kb = static_cast<int>((d + BK - 1) / BK);
-    for (int64_t c = 0; c < n_chunks; ++c) {
-        const int64_t tok0 = c * T_chunk;
-        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
-        const int64_t cg = chunk_index_base + c;
-        for (int64_t i = 0; i < P; ++i) {
-            const int64_t q = ((cg - i) % P + P) % P;                  // Algorithm 3: q = (r - i) mod P
-            const int64_t v_lo = q * block_v;
-            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
-            GemmParams p{};
-            p.m_tiles = (rows + BM - 1) / BM;
-            p.n_tiles = (cols + BN_VOCAB - 1) / BN_VOCAB;
-            p.num_kb = num_kb;
-            p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * d);
-            p.a_mn0 = static_cast<int>(tok0); p.a_k0 = 0;
-            p.b_mn0 = static_cast<int>(v_lo); p.b_k0 = 0;
-            p.rows_valid = rows; p.cols_valid = cols;
-            p.v_lo = static_cast<int>(v_lo);
-            p.labels = labels + tok0;
-            p.ignore_index = ignore_index; p.V = static_cast<int>(V);
-            p.pm = pm; p.pz = pz; p.ylab = ylab; p.part_ld = static_cast<int>(T_chunk);
-            p.status = status;
-            apply_tuning(p, EPI_FOLD);
-            p.tile_counter = counters.take();
-            if (pair_strip && p.m_tiles >= 2) {
-                if (launch_pair<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW_half, tmH, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
-            } else if (launch_gemm<BN_VOCAB, false, false, EPI_FOLD>(tmH, tmW, tmH, p, st) != cudaSuccess) {
-                return VPCE_CUDA_ERROR;
-            }
-            vpce_merge_kernel<<<(rows + 255) / 256, 256, 0, st>>>(pm, pz, static_cast<int>(T_chunk), p.n_tiles, sm, sz, ylab,
-                                                                  rows, i == 0, i == P - 1, labels + tok0, ignore_index,
-                                                                  static_cast<int>(V), lse + tok0, loss + tok0, status);
-            g_launches.fetch_add(1, std::memory_order_relaxed);
-            if (cudaGetLastError() != cudaSuccess) return VPCE_CUDA_ERROR;
-        }
-    }
-    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
-}
-
 vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels, int64_t T, int64_t d, int64_t V,
                           int64_t block_v, int32_t ignore_index, float* loss, float* lse, int64_t T_chunk,
                           int64_t chunk_index_base, void* workspace, size_t workspace_bytes, void* stream) {
     return forward_impl(H, W, labels, T, d, V, block_v, ignore_index, loss, lse, T_chunk, chunk_index_base, workspace,
                         workspace_bytes, stream, true);
-}
-
-static vpce_status backward_impl(const void* H, const void* W, const int32_t* labels, const float* lse,
-                                 const float* dloss, void* dH, float* dW, int64_t T, int64_t d, int64_t V,
-                                 int64_t block_v, int32_t ignore_index, int64_t T_chunk, int64_t chunk_index_base,
-                                 int accumulate_dW, void* workspace, size_t workspace_bytes, void* stream,
-                                 bool clear_status) {
-    WsLayout L;
-    if (T == 0) {                                                      // empty batch: dW gets no contribution
-        if (!accumulate_dW && dW && V > 0 && d > 0 &&
-            cudaMemsetAsync(dW, 0, static_cast<size_t>(V) * d * 4, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-            return VPCE_CUDA_ERROR;
-        return VPCE_OK;
-    }
-    if (!lse || (!dH && !dW)) return VPCE_INVALID_ARG;                 // either gradient may be left out, not both
-    vpce_status s = check_common(H, W, labels, T, d, V, block_v, T_chunk, chunk_index_base, workspace, workspace_bytes, &L);
-    if (s != VPCE_OK) return s;
-    if (!aligned16(dH) || !aligned16(dW)) return VPCE_UNSUPPORTED;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    int* status = reinterpret_cast<int*>(ws + L.status);
-    float* inv_n = reinterpret_cast<float*>(ws + L.scalars);
-    __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(ws + L.G);
-    float* acc = reinterpret_cast<float*>(ws + L.acc);
-
-    CUtensorMap tmH_k, tmW_k, tmG_k, tmW_mn, tmG_mn, tmH_mn, tmG_st;
-    if (!make_map(&tmG_st, G, T_chunk, block_v, block_v, 64, 32) ||
-        !make_map(&tmH_k, H, T, d, d, BK, BM) || !make_map(&tmW_k, W, V, d, d, BK, BN_VOCAB) ||
-        !make_map(&tmG_k, G, T_chunk, block_v, block_v, BK, BM) || !make_map(&tmW_mn, W, V, d, d, 64, BK) ||
-        !make_map(&tmG_mn, G, T_chunk, block_v, block_v, 64, BK) || !make_map(&tmH_mn, H, T, d, d, 64, BK))
-        return VPCE_CUDA_ERROR;
-
-    if (clear_status) {
-        vpce_clear_status_kernel<<<1, 32, 0, st>>>(status);
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-    }
-    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
-    if (!dloss) {
-        vpce_count_valid_kernel<<<1, 1024, 0, st>>>(labels, T, static_cast<int>(V), ignore_index, inv_n, nullptr, status);
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-    }
-
-    const int bn = pick_bn(d);
-    // CTA-pair variants: half-width B boxes
-    const int pmask = pair_mask();
-    CUtensorMap tmW_khalf, tmW_mn2, tmH_mn2;
-    const bool pair_ok = (bn == 256) && (d % 64 == 0);
-    if (!make_map(&tmW_khalf, W, V, d, d, BK, BN_VOCAB / 2)) return VPCE_CUDA_ERROR;
-    if (pair_ok && (!make_map_mn3d(&tmW_mn2, W, V, d, d, 2) || !make_map_mn3d(&tmH_mn2, H, T, d, d, 2))) return VPCE_CUDA_ERROR;
-    // one-instruction fetch of MN-major operands when the contiguous extent is a multiple of 64
-    const bool mn3d = (d % 64 == 0);
-    if (mn3d) {
-        if (!make_map_mn3d(&tmW_mn, W, V, d, d, bn / 64) || !make_map_mn3d(&tmH_mn, H, T, d, d, bn / 64) ||
-            !make_map_mn3d(&tmG_mn, G, T_chunk, block_v, block_v, BM / 64))
-            return VPCE_CUDA_ERROR;
-    }
-    const int64_t P = (V + block_v - 1) / block_v;
-    const int64_t n_chunks = (T + T_chunk - 1) / T_chunk;
-    for (int64_t c = 0; c < n_chunks; ++c) {
-        const int64_t tok0 = c * T_chunk;
-        const int rows = static_cast<int>((T - tok0) < T_chunk ? (T - tok0) : T_chunk);
-        const int64_t cg = chunk_index_base + c;
-        for (int64_t i = 0; i < P; ++i) {
-            const int64_t q = ((cg - i) % P + P) % P;
-            const int64_t v_lo = q * block_v;
-            const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
-            const int strip_tiles_n = (cols + BN_VOCAB - 1) / BN_VOCAB;
-            // (1) recompute the strip and form the residual G (bf16) in the workspace
-            GemmParams p{};
-            p.m_tiles = (rows + BM - 1) / BM;
-            p.n_tiles = strip_tiles_n;
-            p.num_kb = static_cast<int>((d + BK - 1) / BK);
-            p.group_n = pick_group_n(p.n_tiles, 2.0 * cols * d);
-            p.a_mn0 = static_cast<int>(tok0); p.b_mn0 = static_cast<int>(v_lo);
-            p.rows_valid = rows; p.cols_valid = cols;
-            p.v_lo = static_cast<int>(v_lo);
-            p.labels = labels + tok0; p.lse = lse + tok0; p.dloss = dloss ? dloss + tok0 : nullptr;
-            p.inv_n_valid = inv_n; p.ignore_index = ignore_index; p.V = static_cast<int>(V);
-            p.G = G; p.g_ld = static_cast<int>(block_v); p.g_rows = static_cast<int>(T_chunk);
-            p.status = status;
-            apply_tuning(p, EPI_RESID);
-            p.tile_counter = counters.take();
-            if ((pmask & 1) && p.m_tiles >= 2) {
-                if (launch_pair<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_khalf, tmG_st, p, st) != cudaSuccess) return VPCE_CUDA_ERROR;
-            } else if (launch_gemm<BN_VOCAB, false, false, EPI_RESID>(tmH_k, tmW_k, tmG_st, p, st) != cudaSuccess) {
-                return VPCE_CUDA_ERROR;
-            }
-            const int k_cols = strip_tiles_n * BN_VOCAB;               // columns of G written by step (1)
-            const int m_rows = p.m_tiles * BM;                         // rows of G written by step (1)
-            // (2) dH_c += G W_q : M = tokens, N = d, K = shard vocabulary
-            GemmParams ph{};
-            ph.m_tiles = p.m_tiles;
-            ph.n_tiles = static_cast<int>((d + bn - 1) / bn);
-            ph.num_kb = k_cols / BK;
-            ph.group_n = pick_group_n(ph.n_tiles, 2.0 * k_cols * d);
-            ph.a_mn0 = 0; ph.a_k0 = 0;
-            ph.b_mn0 = 0; ph.b_k0 = static_cast<int>(v_lo);
-            ph.rows_valid = rows; ph.cols_valid = static_cast<int>(d);
-            ph.acc = acc; ph.acc_ld = static_cast<int>(d);
-            ph.dH = dH ? static_cast<__nv_bfloat16*>(dH) + tok0 * d : nullptr; ph.out_ld = static_cast<int>(d);
-            ph.first = (i == 0); ph.last = (i == P - 1);
-            ph.status = status;
-            ph.b_3d = mn3d;
-            ph.n_cut = pick_n_cut((ph.m_tiles + 1) / 2, ph.n_tiles, num_sms() / 2);
-            apply_tuning(ph, EPI_DH);
-            ph.tile_counter = counters.take();
-            if (!dH) {
-                // input gradient not wanted
-            } else if ((pmask & 2) && pair_ok && ph.m_tiles >= 2) {
-                if (launch_pair<256, false, true, EPI_DH>(tmG_k, tmW_mn2, tmG_k, ph, st) != cudaSuccess) return VPCE_CUDA_ERROR;
-            } else if (launch_grad<false, true, EPI_DH>(bn, tmG_k, tmW_mn, ph, st) != cudaSuccess) {
-                return VPCE_CUDA_ERROR;
-            }
-            // (3) dW_q += G^T H_c : M = shard vocabulary, N = d, K = chunk tokens
-            GemmParams pw{};
-            pw.m_tiles = (cols + BM - 1) / BM;
-            pw.n_tiles = ph.n_tiles;
-            pw.num_kb = m_rows / BK;
-            pw.group_n = pick_group_n(pw.n_tiles, 2.0 * m_rows * d);
-            pw.a_mn0 = 0; pw.a_k0 = 0;
-            pw.b_mn0 = 0; pw.b_k0 = static_cast<int>(tok0);
-            pw.rows_valid = cols; pw.cols_valid = static_cast<int>(d);
-            if (!dW) continue;                                         // weight gradient not wanted
-            pw.dW = dW + v_lo * d; pw.out_ld = static_cast<int>(d);
-            pw.accumulate = (accumulate_dW != 0) || (c > 0);
-            pw.status = status;
-            pw.a_3d = mn3d; pw.b_3d = mn3d;
-            pw.n_cut = pick_n_cut((pw.m_tiles + 1) / 2, pw.n_tiles, num_sms() / 2);
-            apply_tuning(pw, EPI_DW);
-            pw.tile_counter = counters.take();
-            if ((pmask & 4) && pair_ok && pw.m_tiles >= 2) {
-                if (launch_pair<256, true, true, EPI_DW>(tmG_mn, tmH_mn2, tmG_mn, pw, st) != cudaSuccess) return VPCE_CUDA_ERROR;
-            } else if (launch_grad<true, true, EPI_DW>(bn, tmG_mn, tmH_mn, pw, st) != cudaSuccess) {
-                return VPCE_CUDA_ERROR;
-            }
-        }
-    }
-    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
 }
 
 vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse, const float* dloss,
@@ -570,6 +632,85 @@ vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, 
                            size_t workspace_bytes, void* stream) {
     return backward_impl(H, W, labels, lse, dloss, dH, dW, T, d, V, block_v, ignore_index, T_chunk, chunk_index_base,
                          accumulate_dW, workspace, workspace_bytes, stream, true);
+}
+
+// ---- single meetings for a ring driver (Algorithm 3 across devices)
+size_t vp_ce_meeting_workspace_bytes(int64_t N, int64_t d, int64_t shard_rows) {
+    if (N <= 0 || shard_rows <= 0) return 0;
+    WsLayout L;
+    return ws_layout(align_up(N, BM), d, align_up(shard_rows, BN_VOCAB), &L) ? L.total : 0;
+}
+
+vpce_status vp_ce_meeting_forward(const void* X, const void* W_shard, const int32_t* targets, int64_t N, int64_t d,
+                                  int64_t shard_rows, int64_t v_lo, int64_t V, int32_t ignore_index, float* state,
+                                  int first, int last, float* loss, float* lse, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+    if (!X || !W_shard || !targets || !state || !workspace) return VPCE_INVALID_ARG;
+    if (N <= 0 || d <= 0 || shard_rows <= 0 || v_lo < 0 || V <= 0 || v_lo + shard_rows > V) return VPCE_INVALID_ARG;
+    if (last && (!loss || !lse)) return VPCE_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(W_shard) || !aligned16(workspace)) return VPCE_UNSUPPORTED;
+    if (N >= (1ll << 31) || V >= (1ll << 31)) return VPCE_UNSUPPORTED;
+    WsLayout L;
+    const int64_t n_pad = align_up(N, BM);
+    if (!ws_layout(n_pad, d, align_up(shard_rows, BN_VOCAB), &L)) return VPCE_UNSUPPORTED;
+    if (workspace_bytes < L.total) return VPCE_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    FoldCtx c;
+    if (!make_fold_ctx(&c, X, N, W_shard, shard_rows, d)) return VPCE_CUDA_ERROR;
+    c.status = reinterpret_cast<int*>(ws + L.status);
+    c.sm = state; c.sz = state + N; c.ylab = state + 2 * N;              // the state is the caller's: it may travel
+    c.pm = reinterpret_cast<float*>(ws + L.pm);
+    c.pz = reinterpret_cast<float*>(ws + L.pz);
+    c.part_ld = static_cast<int>(n_pad);
+    c.ignore_index = ignore_index; c.V = static_cast<int>(V);
+    if (first) {                                                       // a batch's first meeting starts a clean status word
+        vpce_clear_status_kernel<<<1, 32, 0, st>>>(c.status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
+    if (fold_meeting(c, 0, static_cast<int>(N), 0, static_cast<int>(shard_rows), static_cast<int>(v_lo), targets, first != 0,
+                     last != 0, lse, loss, counters, st) != cudaSuccess)
+        return VPCE_CUDA_ERROR;
+    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
+}
+
+vpce_status vp_ce_meeting_backward(const void* X, const void* W_shard, const int32_t* targets, const float* lse,
+                                   const float* dloss, int64_t N, int64_t d, int64_t shard_rows, int64_t v_lo, int64_t V,
+                                   int32_t ignore_index, int phases, float* dX_acc, int first, int last, void* dX,
+                                   float* dW_shard, int accumulate_dW, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+    if (!X || !W_shard || !targets || !lse || !dloss || !workspace) return VPCE_INVALID_ARG;
+    if (N <= 0 || d <= 0 || shard_rows <= 0 || v_lo < 0 || V <= 0 || v_lo + shard_rows > V) return VPCE_INVALID_ARG;
+    if (phases <= 0 || phases > 7) return VPCE_INVALID_ARG;
+    if ((phases & PHASE_INPUT_GRAD) && ((!last && !dX_acc) || (last && !dX) || (!first && !dX_acc))) return VPCE_INVALID_ARG;
+    if ((phases & PHASE_WEIGHT_GRAD) && !dW_shard) return VPCE_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(W_shard) || !aligned16(workspace) || !aligned16(dX_acc) || !aligned16(dX) ||
+        !aligned16(dW_shard))
+        return VPCE_UNSUPPORTED;
+    if (N >= (1ll << 31) || V >= (1ll << 31)) return VPCE_UNSUPPORTED;
+    WsLayout L;
+    const int64_t n_pad = align_up(N, BM), s_pad = align_up(shard_rows, BN_VOCAB);
+    if (!ws_layout(n_pad, d, s_pad, &L)) return VPCE_UNSUPPORTED;
+    if (workspace_bytes < L.total) return VPCE_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    GradCtx c;
+    if (!make_grad_ctx(&c, X, N, W_shard, shard_rows, d, reinterpret_cast<__nv_bfloat16*>(ws + L.G), n_pad, s_pad))
+        return VPCE_CUDA_ERROR;
+    c.status = reinterpret_cast<int*>(ws + L.status);
+    c.inv_n = reinterpret_cast<float*>(ws + L.scalars);
+    c.ignore_index = ignore_index; c.V = static_cast<int>(V);
+    if (first && (phases & PHASE_RESIDUAL)) {
+        vpce_clear_status_kernel<<<1, 32, 0, st>>>(c.status);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
+    if (grad_meeting(c, phases, 0, static_cast<int>(N), 0, static_cast<int>(shard_rows), static_cast<int>(v_lo), targets, lse,
+                     dloss, first != 0, last != 0, dX_acc, static_cast<__nv_bfloat16*>(dX), dW_shard, accumulate_dW != 0,
+                     counters, st) != cudaSuccess)
+        return VPCE_CUDA_ERROR;
+    return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
 }
 
 vpce_status vp_ce_mean_loss(const float* loss, const int32_t* labels, int64_t T, int64_t V, int32_t ignore_index,

@@ -103,7 +103,9 @@ __device__ __forceinline__ void epilogue_fold(const GemmParams& p, int mt, int n
     const int grow = mt * BM + row;                             // row within the chunk
     const bool row_ok = grow < p.rows_valid;
     const int label = row_ok ? p.labels[grow] : -1;
-    const int lrel = label - (p.v_lo + nt * BN_VOCAB);          // target column relative to the tile
+    // target column relative to the tile; a target beyond the shard's last valid column belongs to another shard
+    // (its padded column here holds no logit)
+    const int lrel = (label - p.v_lo < p.cols_valid) ? label - (p.v_lo + nt * BN_VOCAB) : -1;
     float m = NEG_INF, z = 0.f, yl = 0.f;
     bool hit = false;
 #pragma unroll 1
