@@ -31,6 +31,12 @@ from .binding import (  # noqa: F401
     vp_ce_mean_loss_grad,
     vp_ce_status_string,
     vp_ce_workspace_bytes,
+    osadamw_create,
+    osadamw_destroy,
+    osadamw_staging_bytes,
+    osadamw_step,
+    osadamw_update_device,
+    osadamw_wait,
 )
 
 

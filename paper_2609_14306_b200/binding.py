@@ -83,6 +83,19 @@ def load_library() -> ctypes.CDLL:
     lib.vp_ce_set_wait_limit_ns.argtypes = [i64]
     lib.vp_ce_debug_drop_copy.restype = ctypes.c_int
     lib.vp_ce_debug_drop_copy.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    f32 = ctypes.c_float
+    lib.osadamw_staging_bytes.restype = sz
+    lib.osadamw_staging_bytes.argtypes = [i64, ctypes.c_int]
+    lib.osadamw_create.restype = ctypes.c_int
+    lib.osadamw_create.argtypes = [ctypes.POINTER(vp), i64, ctypes.c_int, vp, sz]
+    lib.osadamw_destroy.restype = ctypes.c_int
+    lib.osadamw_destroy.argtypes = [vp]
+    lib.osadamw_step.restype = ctypes.c_int
+    lib.osadamw_step.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, f32, f32, f32, f32, f32, i64, vp]
+    lib.osadamw_wait.restype = ctypes.c_int
+    lib.osadamw_wait.argtypes = [vp]
+    lib.osadamw_update_device.restype = ctypes.c_int
+    lib.osadamw_update_device.argtypes = [vp, vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
     lib.vp_ce_profile_enable.restype = None
     lib.vp_ce_profile_enable.argtypes = [ctypes.c_int]
     lib.vp_ce_profile_collect.restype = ctypes.c_int
@@ -369,3 +382,60 @@ def vp_ce_backward_f32(H, W, labels, lse, dloss, dH, dW, block_v: int, ignore_in
             T, d, V, int(block_v), int(ignore_index), int(T_chunk), int(chunk_index_base),
             1 if accumulate_dW else 0,
             _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream, H)))
+
+
+# --------------------------------------------------------------------------- bucket-streamed AdamW (stream_adamw.h)
+def osadamw_staging_bytes(bucket_params: int, slots: int) -> int:
+    return int(load_library().osadamw_staging_bytes(int(bucket_params), int(slots)))
+
+
+def osadamw_create(bucket_params: int, slots: int, staging) -> int:
+    """Creates a pipeline over the caller's device staging buffer (uint8 CUDA tensor); returns the handle."""
+    import torch
+    lib = load_library()
+    handle = ctypes.c_void_p()
+    with _on_device(staging):
+        _check(lib.osadamw_create(ctypes.byref(handle), int(bucket_params), int(slots),
+                                  _ptr(staging, torch.uint8, "staging"), staging.numel()))
+    return int(handle.value)
+
+
+def osadamw_destroy(handle: int) -> None:
+    _check(load_library().osadamw_destroy(ctypes.c_void_p(handle)))
+
+
+def osadamw_step(handle: int, master, m, v, grad, w_bf16, lr: float, beta1: float, beta2: float, eps: float,
+                 weight_decay: float, step: int, bucket_offsets=None, stream=None) -> None:
+    """One optimizer step over HOST fp32 state (CPU tensors, ideally pinned) and the DEVICE bf16 working weight;
+    asynchronous, see osadamw_wait."""
+    import torch
+    lib = load_library()
+    n = master.numel()
+    offs, nb = None, 0
+    if bucket_offsets is not None:
+        offs = (ctypes.c_int64 * len(bucket_offsets))(*[int(o) for o in bucket_offsets])
+        nb = len(bucket_offsets) - 1
+    with _on_device(w_bf16):
+        _check(lib.osadamw_step(
+            ctypes.c_void_p(handle), _host_ptr(master, torch.float32, "master", n), _host_ptr(m, torch.float32, "m", n),
+            _host_ptr(v, torch.float32, "v", n), _host_ptr(grad, torch.float32, "grad", n),
+            _ptr(w_bf16, torch.bfloat16, "w_bf16", n), n, offs, nb,
+            float(lr), float(beta1), float(beta2), float(eps), float(weight_decay), int(step),
+            _stream_ptr(stream, w_bf16)))
+
+
+def osadamw_wait(handle: int) -> None:
+    _check(load_library().osadamw_wait(ctypes.c_void_p(handle)))
+
+
+def osadamw_update_device(p, m, v, g, w_bf16, lr: float, beta1: float, beta2: float, eps: float, weight_decay: float,
+                          step: int, stream=None) -> None:
+    """The fused AdamW update + bf16 refresh on device-resident fp32 state (in place)."""
+    import torch
+    lib = load_library()
+    n = p.numel()
+    with _on_device(p):
+        _check(lib.osadamw_update_device(
+            _ptr(p, torch.float32, "p"), _ptr(m, torch.float32, "m", n), _ptr(v, torch.float32, "v", n),
+            _ptr(g, torch.float32, "g", n), _ptr(w_bf16, torch.bfloat16, "w_bf16", n), n,
+            float(lr), float(beta1), float(beta2), float(eps), float(weight_decay), int(step), _stream_ptr(stream, p)))

@@ -16,7 +16,7 @@ def declared_functions():
     for fn in sorted(os.listdir(inc)):
         if fn.endswith(".h"):
             text = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, fn)).read(), flags=re.S)
-            names += re.findall(r"\b(vp_ce_\w+)\s*\(", text)
+            names += re.findall(r"\b((?:vp_ce|osadamw)_\w+)\s*\(", text)
     return sorted(set(names))
 
 
@@ -25,7 +25,8 @@ def test_library_exports_every_declared_symbol():
     lib = vp.load_library()
     names = declared_functions()
     assert {"vp_ce_forward", "vp_ce_backward", "vp_ce_workspace_bytes", "vp_ce_mean_loss",
-            "vp_ce_device_status", "vp_ce_status_string"} <= set(names)
+            "vp_ce_device_status", "vp_ce_status_string", "vp_ce_meeting_forward", "vp_ce_meeting_backward",
+            "osadamw_create", "osadamw_step", "osadamw_wait", "osadamw_update_device"} <= set(names)
     raw = ctypes.CDLL(vp.library_path())
     for n in names:
         assert hasattr(raw, n), n
@@ -68,3 +69,10 @@ def test_wait_limit_and_test_hook_arguments():
             vp.vp_ce_debug_drop_copy(*bad)
     vp.vp_ce_debug_drop_copy(2, 3, 3)
     vp.vp_ce_debug_drop_copy(-1)                              # disarm
+
+
+def test_streamed_adamw_staging_size():
+    # pure host arithmetic: 16 bytes per parameter and slot (p, m, v, g in fp32), arrays padded to 256 bytes
+    assert vp.osadamw_staging_bytes(1 << 20, 2) == 2 * 4 * (1 << 20) * 4
+    assert vp.osadamw_staging_bytes(100, 3) == 3 * 4 * 128 * 4
+    assert vp.osadamw_staging_bytes(0, 2) == 0 and vp.osadamw_staging_bytes(100, 0) == 0
