@@ -453,6 +453,119 @@ def measure(ctx, w, dtype, steps, warmup, t_chunk=0, with_e2e=True, with_cpu_bas
     return out
 
 
+def link_peaks(dev, nbytes=1 << 30):
+    """Measured pinned-memory copy bandwidth of the host link, GB/s: each direction alone and both at once
+    (plain cudaMemcpyAsync through torch, best of 3).  The yard-stick the streamed optimizer is measured against."""
+    import torch
+    h_in = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    h_out = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    d_in = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    d_out = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+
+    def run(h2d, d2h):
+        best = 1e30
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            if h2d:
+                with torch.cuda.stream(s1):
+                    d_in.copy_(h_in, non_blocking=True)
+            if d2h:
+                with torch.cuda.stream(s2):
+                    h_out.copy_(d_out, non_blocking=True)
+            torch.cuda.synchronize()
+            best = min(best, time.perf_counter() - t0)
+        return nbytes / best / 1e9
+    return {"h2d_alone": run(True, False), "d2h_alone": run(False, True), "each_direction_when_both_run": run(True, True)}
+
+
+def measure_adamw(ctx, n_params, bucket, slots, steps, warmup):
+    """OffloadStreamAdamW (the paper's other named GPU kernel): one optimizer step over `n_params` parameters whose fp32
+    master weights, moments and gradients live in pinned HOST memory, streamed through `slots` device slots of `bucket`
+    parameters.  Bound by the host link: 16 bytes in and 12 bytes out per parameter."""
+    import torch
+    import paper_2609_14306_b200 as vp
+    dev = ctx.dev
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+    g = torch.Generator().manual_seed(7)
+    host = [torch.empty(n_params, dtype=torch.float32).pin_memory() for _ in range(4)]      # master, m, v, grad
+    chunk = 1 << 24
+    for a in range(0, n_params, chunk):                                                     # seeded, synthetic state
+        b = min(n_params, a + chunk)
+        host[0][a:b] = torch.randn(b - a, generator=g) * 0.02
+        host[1][a:b] = torch.randn(b - a, generator=g) * 1e-3
+        host[2][a:b] = torch.randn(b - a, generator=g).square_() * 1e-6
+        host[3][a:b] = torch.randn(b - a, generator=g) * 1e-2
+    sample = [h[: 1 << 22].clone() for h in host]                                           # the CPU leg's inputs (before any step)
+    w = torch.empty(n_params, dtype=torch.bfloat16, device=dev)
+    staging = torch.empty(vp.osadamw_staging_bytes(bucket, slots), dtype=torch.uint8, device=dev)
+    h = vp.osadamw_create(bucket, slots, staging)
+    sampler = ClockSampler(ctx.local_rank)
+    try:
+        t = 0
+        for _ in range(warmup):
+            t += 1
+            vp.osadamw_step(h, *host, w, step=t, **hp)
+        vp.osadamw_wait(h)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            t += 1
+            vp.osadamw_step(h, *host, w, step=t, **hp)
+        vp.osadamw_wait(h)                       # the host state is complete: this is the end of an optimizer step
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+    finally:
+        vp.osadamw_destroy(h)
+    clocks = sampler.stop()
+    # the update kernel alone on device-resident state (what the pipeline hides behind the copies)
+    nk = min(n_params, 1 << 26)
+    dstate = [torch.randn(nk, device=dev) * 1e-2 for _ in range(4)]
+    dstate[2].square_()
+    for _ in range(3):
+        vp.osadamw_update_device(*dstate, w[:nk], step=1, **hp)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(10):
+        vp.osadamw_update_device(*dstate, w[:nk], step=2 + i, **hp)
+    e1.record()
+    torch.cuda.synchronize()
+    k_ms = e0.elapsed_time(e1) / 10
+    del dstate, staging, w
+    torch.cuda.empty_cache()
+    link = link_peaks(dev)
+    peaks, peak_src = load_peaks()
+    in_gbs = 16.0 * n_params / (ms / 1e3) / 1e9
+    # the oracle as it stands on a bounded sample (float64, one pass over 4 Mi parameters)
+    from oracle import adamw_oracle as ao
+    t0 = time.perf_counter()
+    ao.adamw_step(*(x.numpy() for x in sample), 1, **hp)
+    cpu_dt = time.perf_counter() - t0
+    return {
+        "metric": "OffloadStreamAdamW optimizer step, parameters/s (host-resident fp32 state)", "value": n_params / (ms / 1e3),
+        "unit": "parameters/s", "ms_per_step": ms, "steps": steps, "warmup": warmup, "dtype": "f32", "data": "synthetic",
+        "higher_is_better": True,
+        "config": {"workload": "osadamw", "parameters": n_params, "bucket_params": bucket, "slots": slots,
+                   "buckets": -(-n_params // bucket), "staging_bytes": vp.osadamw_staging_bytes(bucket, slots),
+                   "host_memory": "pinned", "bytes_in_per_param": 16, "bytes_out_per_param": 12},
+        "roofline": {"bound": "host-link", "achieved": in_gbs, "peak": link["each_direction_when_both_run"], "unit": "GB/s",
+                     "frac": in_gbs / link["each_direction_when_both_run"],
+                     "peak_kind": "pinned cudaMemcpyAsync host-to-device bandwidth while a device-to-host copy runs, "
+                                  "measured in this process (no such figure is in the measured-peaks file)",
+                     "traffic": None, "link_gbs": link, "out_gbs": 12.0 * n_params / (ms / 1e3) / 1e9},
+        "update_kernel": {"parameters": nk, "ms": k_ms, "gbs": 30.0 * nk / (k_ms / 1e3) / 1e9,
+                          "hbm_peak_gbs": peaks["hbm_gbs"], "frac_of_hbm_peak": 30.0 * nk / (k_ms / 1e3) / 1e9 / peaks["hbm_gbs"],
+                          "bytes_per_param": 30, "peak_source": peak_src},
+        "cpu_baseline": {"value": sample[0].numel() / cpu_dt, "unit": "parameters/s", "cores": os.cpu_count(), "kind": "oracle",
+                         "sample": f"float64 AdamW step over the first {sample[0].numel()} parameters, {cpu_dt:.2f} s wall clock"},
+        "clocks": clocks,
+    }
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -471,6 +584,7 @@ def main():
                     help="skip the extra measured blocks (the other target configuration, the paper's shape in TF32)")
     ap.add_argument("--no-yardstick", action="store_true", help="skip the cuBLAS context measurement")
     ap.add_argument("--profile-in-timed-region", type=int, default=1)
+    ap.add_argument("--adamw", default="", help="measure only the streamed AdamW: parameters,bucket,slots (e.g. 268435456,100000000,2)")
     args = ap.parse_args()
 
     from synth_inputs import PROFILE_WORKLOADS, WORKLOADS
@@ -492,6 +606,12 @@ def main():
     ctx = Ctx()
     vp.load_library()          # raises if the CUDA library is missing: there is no fallback
 
+    if args.adamw:
+        n_, b_, s_ = (int(x) for x in args.adamw.split(","))
+        if ctx.rank == 0:
+            print(json.dumps(measure_adamw(ctx, n_, b_, s_, max(1, args.steps), args.warmup)), flush=True)
+        ctx.close()
+        return
     prof_on = bool(args.profile_in_timed_region)
     out = measure(ctx, w, args.dtype, args.steps, args.warmup, t_chunk=args.t_chunk, with_e2e=not args.no_e2e,
                   with_cpu_baseline=not args.no_cpu_baseline, with_yardstick=not args.no_yardstick, prof_on=prof_on)
@@ -505,6 +625,7 @@ def main():
                     with_yardstick=not args.no_yardstick, prof_on=prof_on),
             measure(ctx, PROFILE_WORKLOADS["papershape"], "tf32", 3, 3, with_e2e=False, with_cpu_baseline=False,
                     prof_on=prof_on),
+            measure_adamw(ctx, n_params=1 << 28, bucket=1 << 25, slots=2, steps=3, warmup=2),
         ]
     if ctx.rank == 0:
         print(json.dumps(out), flush=True)
