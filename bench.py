@@ -39,6 +39,8 @@ FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_g
 NCU_DRAM_BYTES_PER_LAUNCH = {
     ("bf16", 2880, 8192, 16384): {"fwd_strip_fold": 156e6, "bwd_strip_residual": 462e6, "dH_gemm": 776e6,
                                   "dW_gemm": 964e6},
+    ("bf16", 7168, 8192, 8192): {"fwd_strip_fold": 638e6, "bwd_strip_residual": 930e6, "dH_gemm": 1093e6,
+                                 "dW_gemm": 1087e6},
 }
 # Token chunk used by the timed launch configuration (a call argument of the library).
 BENCH_T_CHUNK = {"tiny": 512, "mid": 4096, "moe120b": 16384, "moe667b": 8192, "longctx": 16384}
@@ -56,7 +58,7 @@ def load_peaks():
 # --------------------------------------------------------------------------- clocks sampler
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index: int):
         self.rows = []
@@ -92,8 +94,15 @@ class ClockSampler:
         mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        watts = []
+        for r in self.rows:
+            try:
+                watts.append(float(r[6]))
+            except (IndexError, ValueError):
+                pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+                "reasons": reasons, "samples": len(sm),
+                "power_w_median": statistics.median(watts) if watts else None}
 
 
 # --------------------------------------------------------------------------- CPU oracle leg
@@ -213,14 +222,18 @@ def cublas_yardstick(w, T_chunk, dev, seconds=1.0):
             fn()
         e1.record(); torch.cuda.synchronize()
         out[name] = flops * n / (e0.elapsed_time(e1) / 1e3) / 1e12
-    # the three in the order of a backward meeting, interleaved, as the step runs them
-    n = max(3, int(seconds * 1e3 / (3 * flops / (out["strip"] * 1e12) * 1e3)))
+    # the three in the order of a backward meeting, interleaved, as the step runs them (clocks and power sampled)
+    n = max(3, int(2 * seconds * 1e3 / (3 * flops / (out["strip"] * 1e12) * 1e3)))
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    time.sleep(0.3)
     e0.record()
     for _ in range(n):
         for fn in cases.values():
             fn()
     e1.record(); torch.cuda.synchronize()
     out["interleaved"] = 3 * flops * n / (e0.elapsed_time(e1) / 1e3) / 1e12
+    out["interleaved_clocks"] = sampler.stop()
     return out
 
 
