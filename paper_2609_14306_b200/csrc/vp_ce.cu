@@ -280,12 +280,13 @@ int pick_bn(int64_t d) {
 }
 
 template <bool A_MN, bool B_MN, int EPI>
-cudaError_t launch_grad(int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+cudaError_t launch_grad(int bn, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, const GemmParams& p,
+                        cudaStream_t st) {
     switch (bn) {
-        case 256: return launch_gemm<256, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
-        case 192: return launch_gemm<192, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
-        case 128: return launch_gemm<128, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
-        default:  return launch_gemm<64, A_MN, B_MN, EPI>(tmA, tmB, tmA, p, st);
+        case 256: return launch_gemm<256, A_MN, B_MN, EPI>(tmA, tmB, tmC, p, st);
+        case 192: return launch_gemm<192, A_MN, B_MN, EPI>(tmA, tmB, tmC, p, st);
+        case 128: return launch_gemm<128, A_MN, B_MN, EPI>(tmA, tmB, tmC, p, st);
+        default:  return launch_gemm<64, A_MN, B_MN, EPI>(tmA, tmB, tmC, p, st);
     }
 }
 
@@ -446,7 +447,11 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
     const int m_rows = m_tiles * BM;                           // rows of G written by the residual phase
     const int grad_n_tiles = (d + c.bn - 1) / c.bn;
     if (phases & PHASE_INPUT_GRAD) {
-        // dX += G W_q : M = tokens, N = d, K = shard vocabulary
+        // dX += G W_q : M = tokens, N = d, K = shard vocabulary.  The fp32 running sum lives in `acc`; the tile is
+        // stored on the batch's first meeting and added (TMA reduction) afterwards; rows past the batch are dropped
+        // by the output map's extent.  After the last meeting the sum is rounded to the bf16 output.
+        CUtensorMap tmAcc;
+        if (!make_map(&tmAcc, acc, rows, d, d, 32, 32, 4)) return cudaErrorInvalidValue;
         GemmParams ph{};
         ph.m_tiles = m_tiles;
         ph.n_tiles = grad_n_tiles;
@@ -455,20 +460,27 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         ph.a_mn0 = 0; ph.a_k0 = 0;
         ph.b_mn0 = 0; ph.b_k0 = w_row0;
         ph.rows_valid = rows; ph.cols_valid = d;
-        ph.acc = acc; ph.acc_ld = d;
-        ph.dH = dX; ph.out_ld = d;
-        ph.first = first; ph.last = last;
+        ph.c_row0 = 0; ph.accumulate = first ? 0 : 1;
         ph.status = c.status;
         ph.b_3d = c.mn3d;
         ph.n_cut = pick_n_cut((ph.m_tiles + 1) / 2, ph.n_tiles, num_sms() / 2);
         apply_tuning(ph, EPI_DH);
         ph.tile_counter = counters.take();
-        if ((c.pmask & 2) && c.pair_ok && ph.m_tiles >= 2) e = launch_pair<256, false, true, EPI_DH>(c.tmG_k, c.tmW_mn2, c.tmG_k, ph, st);
-        else e = launch_grad<false, true, EPI_DH>(c.bn, c.tmG_k, c.tmW_mn, ph, st);
+        if ((c.pmask & 2) && c.pair_ok && ph.m_tiles >= 2) e = launch_pair<256, false, true, EPI_DH>(c.tmG_k, c.tmW_mn2, tmAcc, ph, st);
+        else e = launch_grad<false, true, EPI_DH>(c.bn, c.tmG_k, c.tmW_mn, tmAcc, ph, st);
         if (e != cudaSuccess) return e;
+        if (last && dX) {
+            const long n8 = static_cast<long>(rows) * d / 8;
+            const long blocks = (n8 + 255) / 256;
+            vpce_acc_to_bf16_kernel<<<static_cast<unsigned>(blocks < 148 * 8 ? blocks : 148 * 8), 256, 0, st>>>(acc, dX, n8);
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        }
     }
     if (phases & PHASE_WEIGHT_GRAD) {
-        // dW_q += G^T X : M = shard vocabulary, N = d, K = batch tokens
+        // dW_q += G^T X : M = shard vocabulary, N = d, K = batch tokens; stored or added like the input gradient
+        CUtensorMap tmDW;
+        if (!make_map(&tmDW, dW_q, cols, d, d, 32, 32, 4)) return cudaErrorInvalidValue;
         GemmParams pw{};
         pw.m_tiles = (cols + BM - 1) / BM;
         pw.n_tiles = grad_n_tiles;
@@ -477,15 +489,14 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         pw.a_mn0 = 0; pw.a_k0 = 0;
         pw.b_mn0 = 0; pw.b_k0 = x_row0;
         pw.rows_valid = cols; pw.cols_valid = d;
-        pw.dW = dW_q; pw.out_ld = d;
-        pw.accumulate = accumulate_dW;
+        pw.c_row0 = 0; pw.accumulate = accumulate_dW ? 1 : 0;
         pw.status = c.status;
         pw.a_3d = c.mn3d; pw.b_3d = c.mn3d;
         pw.n_cut = pick_n_cut((pw.m_tiles + 1) / 2, pw.n_tiles, num_sms() / 2);
         apply_tuning(pw, EPI_DW);
         pw.tile_counter = counters.take();
-        if ((c.pmask & 4) && c.pair_ok && pw.m_tiles >= 2) e = launch_pair<256, true, true, EPI_DW>(c.tmG_mn, c.tmX_mn2, c.tmG_mn, pw, st);
-        else e = launch_grad<true, true, EPI_DW>(c.bn, c.tmG_mn, c.tmX_mn, pw, st);
+        if ((c.pmask & 4) && c.pair_ok && pw.m_tiles >= 2) e = launch_pair<256, true, true, EPI_DW>(c.tmG_mn, c.tmX_mn2, tmDW, pw, st);
+        else e = launch_grad<true, true, EPI_DW>(c.bn, c.tmG_mn, c.tmX_mn, tmDW, pw, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -683,7 +694,7 @@ vpce_status vp_ce_meeting_backward(const void* X, const void* W_shard, const int
     if (!X || !W_shard || !targets || !lse || !dloss || !workspace) return VPCE_INVALID_ARG;
     if (N <= 0 || d <= 0 || shard_rows <= 0 || v_lo < 0 || V <= 0 || v_lo + shard_rows > V) return VPCE_INVALID_ARG;
     if (phases <= 0 || phases > 7) return VPCE_INVALID_ARG;
-    if ((phases & PHASE_INPUT_GRAD) && ((!last && !dX_acc) || (last && !dX) || (!first && !dX_acc))) return VPCE_INVALID_ARG;
+    if ((phases & PHASE_INPUT_GRAD) && ((!(first && last) && !dX_acc) || (last && !dX))) return VPCE_INVALID_ARG;
     if ((phases & PHASE_WEIGHT_GRAD) && !dW_shard) return VPCE_INVALID_ARG;
     if (!aligned16(X) || !aligned16(W_shard) || !aligned16(workspace) || !aligned16(dX_acc) || !aligned16(dX) ||
         !aligned16(dW_shard))
@@ -706,8 +717,10 @@ vpce_status vp_ce_meeting_backward(const void* X, const void* W_shard, const int
         g_launches.fetch_add(1, std::memory_order_relaxed);
     }
     CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
+    // a batch whose only meeting this is (first and last) needs no travelling accumulator: the workspace's own serves
+    float* acc = dX_acc ? dX_acc : reinterpret_cast<float*>(ws + L.acc);
     if (grad_meeting(c, phases, 0, static_cast<int>(N), 0, static_cast<int>(shard_rows), static_cast<int>(v_lo), targets, lse,
-                     dloss, first != 0, last != 0, dX_acc, static_cast<__nv_bfloat16*>(dX), dW_shard, accumulate_dW != 0,
+                     dloss, first != 0, last != 0, acc, static_cast<__nv_bfloat16*>(dX), dW_shard, accumulate_dW != 0,
                      counters, st) != cudaSuccess)
         return VPCE_CUDA_ERROR;
     return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;

@@ -15,8 +15,11 @@ constexpr int UMMA_K = 16;       // K per tcgen05.mma for 16-bit inputs
 constexpr int BN_VOCAB = 256;    // vocabulary columns per strip tile
 constexpr int NUM_THREADS = 192;
 constexpr int SMEM_BUDGET = 200 * 1024;    // operand stages
+constexpr int SMEM_BUDGET_STAGED = 193 * 1024;   // operand stages of a kernel that also stages its output tile
 constexpr int SMEM_EXTRA = 2048;           // barriers + alignment slack
-constexpr int G_STAGING_BYTES = 4 * 2 * 4096;   // RESID: per epilogue warp two 32-row x 64-column bf16 boxes
+// Output staging of every epilogue that writes a tile (all but the fold): per epilogue warp two 32-row x 128-byte
+// boxes (64 bf16 or 32 fp32 columns) that leave through TMA stores / reductions.
+constexpr int G_STAGING_BYTES = 4 * 2 * 4096;
 
 enum Epilogue { EPI_FOLD = 0, EPI_RESID = 1, EPI_DH = 2, EPI_DW = 3 };
 
@@ -44,15 +47,9 @@ struct GemmParams {
     __nv_bfloat16* G;                      // [T_chunk][g_ld]
     int g_ld;
     int g_rows;                            // rows of the G workspace (T_chunk)
-    // DH
-    float* acc;                            // [T_chunk][acc_ld] fp32 running dH of the chunk
-    int acc_ld;
-    __nv_bfloat16* dH;                     // chunk base, leading dimension out_ld
-    int first, last;
-    // DW
-    float* dW;                             // shard base (row v_lo), leading dimension out_ld
-    int accumulate;
-    int out_ld;
+    // DH / DW: the fp32 output is described by the launch's third tensor map (boxes of 32 columns x 32 rows)
+    int c_row0;                            // output row of accumulator row 0 of tile 0 (map coordinates)
+    int accumulate;                        // 0: the tile is stored; else it is added to the output (TMA reduction)
     int* status;
     int* tile_counter;                     // zero before the launch; tiles are taken with atomicAdd
     unsigned long long wait_limit_ns;      // every wait inside the kernel gives up after this long
@@ -63,18 +60,17 @@ struct GemmParams {
     int drop_kb, drop_ranks;
 };
 
-template <int BN> struct StageCfg {
+template <int BN, int EPI = EPI_FOLD> struct StageCfg {
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (SMEM_BUDGET / STAGE_BYTES) > 8 ? 8 : (SMEM_BUDGET / STAGE_BYTES);
-    static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
-    // the residual epilogue stages its bf16 tile in shared memory for TMA stores
-    static constexpr int SMEM_TOTAL_STAGED = SMEM_TOTAL + G_STAGING_BYTES;
+    static constexpr int BUDGET = EPI == EPI_FOLD ? SMEM_BUDGET : SMEM_BUDGET_STAGED;
+    static constexpr int STAGES = (BUDGET / STAGE_BYTES) > 8 ? 8 : (BUDGET / STAGE_BYTES);
+    // every epilogue but the fold stages its output tile in shared memory for TMA stores
+    static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA + (EPI == EPI_FOLD ? 0 : G_STAGING_BYTES);
+    static_assert(SMEM_TOTAL <= 227 * 1024, "shared memory per CTA");
 };
-template <int BN, int EPI> constexpr int smem_total() {
-    return EPI == EPI_RESID ? StageCfg<BN>::SMEM_TOTAL_STAGED : StageCfg<BN>::SMEM_TOTAL;
-}
+template <int BN, int EPI> constexpr int smem_total() { return StageCfg<BN, EPI>::SMEM_TOTAL; }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
@@ -247,66 +243,37 @@ __device__ __forceinline__ void epilogue_resid_f32(const GemmParams& p, const CU
     }
 }
 
-// ncol0: first output column of the tile; n_this: its width (columns beyond cols_valid are skipped).
-__device__ __forceinline__ void epilogue_dh(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
-    const int grow = mt * BM + row;
-    const bool row_ok = grow < p.rows_valid;
+// fp32 output tile of the two gradient GEMMs.  Each epilogue warp owns 32 accumulator rows; per 32 columns it fills a
+// 32 x 128-byte box in shared memory (128-byte swizzle: 16-byte chunk q of row r sits at chunk q ^ (r & 7)) and one
+// lane hands it to the TMA unit, either as a store (the first contribution to this output) or as a reduction that ADDS
+// the box to what global memory holds (fp32, done at the L2: the running sum never travels back to the SM).  Global
+// traffic is whole 128-byte lines, and rows or columns outside the output's extent (the tensor map's) are dropped by
+// the TMA unit, so no thread needs a bounds check.  Every output element receives exactly one contribution per launch
+// and launches are ordered by the stream, so the sum's order is fixed.
+// x0: first output column of the tile; y0: output row of this warp's first accumulator row; n_this: tile width.
+__device__ __forceinline__ void epilogue_f32_tile(const CUtensorMap* tmC, uint32_t stage_smem, int x0, int y0, int lane,
+                                                  uint32_t tmem_row, int n_this, bool reduce) {
 #pragma unroll 1
     for (int c = 0; c < (n_this + 31) / 32; ++c) {
-        float v[32];
+        const uint32_t buf = stage_smem + (c & 1) * 4096;
+        if (lane == 0) bulk_wait_read_1();                              // the copy that last read this buffer is done
         __syncwarp();
+        float v[32];
         tmem_ld32(tmem_row + c * 32, v);
         tmem_ld_wait();
-        const int col0 = ncol0 + c * 32;
-        if (row_ok) {
-        float* arow = p.acc + static_cast<size_t>(grow) * p.acc_ld + col0;
-        __nv_bfloat16* orow = p.dH + static_cast<size_t>(grow) * p.out_ld + col0;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {                                  // 8 columns per step
-            if (col0 + 8 * q >= p.cols_valid) break;                   // d is a multiple of 8
-            float* x = v + 8 * q;
-            if (!p.first) {
-                const float4 a0 = __ldcs(reinterpret_cast<const float4*>(arow + 8 * q));      // streamed: read once
-                const float4 a1 = __ldcs(reinterpret_cast<const float4*>(arow + 8 * q + 4));
-                x[0] += a0.x; x[1] += a0.y; x[2] += a0.z; x[3] += a0.w;
-                x[4] += a1.x; x[5] += a1.y; x[6] += a1.z; x[7] += a1.w;
-            }
-            if (p.last) {
-                uint4 o;
-                o.x = pack_bf16x2(x[0], x[1]); o.y = pack_bf16x2(x[2], x[3]);
-                o.z = pack_bf16x2(x[4], x[5]); o.w = pack_bf16x2(x[6], x[7]);
-                __stcs(reinterpret_cast<uint4*>(orow + 8 * q), o);
-            } else {
-                __stcs(reinterpret_cast<float4*>(arow + 8 * q), make_float4(x[0], x[1], x[2], x[3]));
-                __stcs(reinterpret_cast<float4*>(arow + 8 * q + 4), make_float4(x[4], x[5], x[6], x[7]));
-            }
+        for (int q = 0; q < 8; ++q) {
+            uint4 o;
+            o.x = __float_as_uint(v[4 * q]); o.y = __float_as_uint(v[4 * q + 1]);
+            o.z = __float_as_uint(v[4 * q + 2]); o.w = __float_as_uint(v[4 * q + 3]);
+            st_shared_v4(buf + lane * 128 + ((q ^ (lane & 7)) << 4), o);
         }
-        }
-    }
-}
-
-__device__ __forceinline__ void epilogue_dw(const GemmParams& p, int mt, int ncol0, int row, uint32_t tmem_row, int n_this) {
-    const int grow = mt * BM + row;                                    // vocabulary row within the shard
-    const bool row_ok = grow < p.rows_valid;
-#pragma unroll 1
-    for (int c = 0; c < (n_this + 31) / 32; ++c) {
-        float v[32];
+        fence_proxy_async();
         __syncwarp();
-        tmem_ld32(tmem_row + c * 32, v);
-        tmem_ld_wait();
-        const int col0 = ncol0 + c * 32;
-        if (row_ok) {
-        float* orow = p.dW + static_cast<size_t>(grow) * p.out_ld + col0;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {                                  // 4 columns per step
-            if (col0 + 4 * q >= p.cols_valid) break;
-            float4 x = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-            if (p.accumulate) {
-                const float4 a = __ldcs(reinterpret_cast<const float4*>(orow + 4 * q));
-                x.x += a.x; x.y += a.y; x.z += a.z; x.w += a.w;
-            }
-            __stcs(reinterpret_cast<float4*>(orow + 4 * q), x);                     // streamed: not re-read by this launch
-        }
+        if (lane == 0) {
+            if (reduce) tma_reduce_add_2d(tmC, buf, x0 + c * 32, y0);
+            else tma_store_2d(tmC, buf, x0 + c * 32, y0);
+            bulk_commit();
         }
     }
 }
@@ -323,7 +290,7 @@ template <int BN, bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-    using Cfg = StageCfg<BN>;
+    using Cfg = StageCfg<BN, EPI>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr uint32_t TMEM_COLS = (BN > 128) ? 512u : (BN > 64 ? 256u : 128u);
     constexpr uint32_t ACC_STRIDE = TMEM_COLS / 2;
@@ -514,13 +481,13 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t tmem_row = tmem_base + ab * ACC_STRIDE + (static_cast<uint32_t>(quad * 32) << 16);
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh(p, mt, nt * BN, row, tmem_row, tile_n(nt));
-            else epilogue_dw(p, mt, nt * BN, row, tmem_row, tile_n(nt));
+            else epilogue_f32_tile(&tmC, g_staging + (warp - 2) * 8192, nt * BN, p.c_row0 + mt * BM + quad * 32, lane,
+                                   tmem_row, tile_n(nt), p.accumulate != 0);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(ab));
         }
-        if (EPI == EPI_RESID && lane == 0) bulk_wait_all();             // staged stores have landed
+        if (EPI != EPI_FOLD && lane == 0) bulk_wait_all();              // staged stores / reductions have landed
     }
 
     tc_fence_before();
@@ -546,17 +513,18 @@ vpce_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // from the launch's counter and publishes them to both CTAs through a small ring (see below).
 // With TF32 = true the operands are 32-bit floats multiplied as TF32 (kind::tf32, K = 8 per MMA,
 // k-blocks of 32 elements); the 128-byte rows and hence all byte sizes are the same.
-// The residual kernel gives 32 KB of the 227 KB to its store staging; the others use them for a 7th stage.
+// The kernels that write an output tile give 32 KB of the 227 KB to its staging (6 stages); the fold kernel uses them
+// for a 7th stage.
 template <int BN, int EPI = EPI_RESID> struct PairCfg {
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (BN / 2) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int BUDGET = SMEM_BUDGET + (EPI == EPI_RESID ? 0 : 28 * 1024);
+    static constexpr int BUDGET = SMEM_BUDGET + (EPI == EPI_FOLD ? 28 * 1024 : 0);
     static constexpr int STAGES = (BUDGET / STAGE_BYTES) > 8 ? 8 : (BUDGET / STAGE_BYTES);
     static constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_EXTRA;
 };
 template <int BN, int EPI> constexpr int pair_smem_total() {
-    return PairCfg<BN, EPI>::SMEM_TOTAL + (EPI == EPI_RESID ? G_STAGING_BYTES : 0);
+    return PairCfg<BN, EPI>::SMEM_TOTAL + (EPI == EPI_FOLD ? 0 : G_STAGING_BYTES);
 }
 
 template <int BN, bool A_MN, bool B_MN, int EPI, bool TF32 = false>
@@ -815,14 +783,14 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
             else if (EPI == EPI_RESID && TF32) epilogue_resid_f32(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else if (EPI == EPI_DH) epilogue_dh(p, mt, ncol0, row, tmem_row, width);
-            else epilogue_dw(p, mt, ncol0, row, tmem_row, width);
+            else epilogue_f32_tile(&tmC, g_staging + (warp - 2) * 8192, ncol0, p.c_row0 + mt * BM + quad * 32, lane, tmem_row,
+                                   width, p.accumulate != 0);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
             ++it;
         }
-        if (EPI == EPI_RESID && lane == 0) bulk_wait_all();
+        if (EPI != EPI_FOLD && lane == 0) bulk_wait_all();
     }
 
     tc_fence_before();
@@ -911,6 +879,19 @@ __global__ void vpce_mean_loss_kernel(const float* __restrict__ loss, const int3
     if (threadIdx.x == 0) {
         *mean_out = cnts[0] > 0 ? static_cast<float>(sums[0] / cnts[0]) : 0.f;
         *n_valid_out = cnts[0];
+    }
+}
+
+// Rounds the finished fp32 input-gradient accumulator of a chunk to the bf16 output (once per chunk).
+__global__ void vpce_acc_to_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ out, long n8) {
+    const long stride = static_cast<long>(gridDim.x) * blockDim.x;
+    for (long i = static_cast<long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += stride) {
+        const float4 a = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i);
+        const float4 b = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i + 1);
+        uint4 o;
+        o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
+        o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
+        reinterpret_cast<uint4*>(out)[i] = o;
     }
 }
 
