@@ -11,7 +11,7 @@ REPO_DIR = os.path.dirname(PKG_DIR)
 SOURCES = [os.path.join(PKG_DIR, "csrc", "vp_ce.cu"), os.path.join(PKG_DIR, "csrc", "stream_adamw.cu")]
 HEADERS = [os.path.join(REPO_DIR, "include", "vp_ce.h"), os.path.join(REPO_DIR, "include", "stream_adamw.h"),
            os.path.join(PKG_DIR, "csrc", "sm100_ptx.cuh"), os.path.join(PKG_DIR, "csrc", "vp_ce_kernels.cuh"),
-           os.path.join(PKG_DIR, "csrc", "vp_ce_f32.inc")]
+           os.path.join(PKG_DIR, "csrc", "vp_ce_f32.inc"), os.path.join(PKG_DIR, "csrc", "vp_ce_fixup.cuh")]
 LIB_PATH = os.path.join(PKG_DIR, "libvpce.so")
 
 NVCC_FLAGS = [

@@ -37,6 +37,7 @@
 
 #include "vp_ce.h"
 #include "vp_ce_kernels.cuh"
+#include "vp_ce_fixup.cuh"
 
 namespace {
 
@@ -87,10 +88,19 @@ struct CounterPool {
         }
         return base + next++;
     }
+    int* take_n(int k) {                                      // k consecutive zeroed counters
+        if (next + k > NUM_TILE_COUNTERS) {
+            failed = failed || cudaMemsetAsync(base, 0, 4 * NUM_TILE_COUNTERS, st) != cudaSuccess;
+            next = 0;
+        }
+        int* p = base + next;
+        next += k;
+        return p;
+    }
 };
 
 struct WsLayout {
-    size_t status, scalars, counters, sm, sz, ylab, pm, pz, G, acc, total;
+    size_t status, scalars, counters, sm, sz, ylab, pm, pz, G, acc, delta, keys, partials, total;
 };
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -110,6 +120,11 @@ bool ws_layout(int64_t T_chunk, int64_t d, int64_t block_v, WsLayout* L, int g_e
     L->pz = off;      off = align_up(off + 4 * T_chunk * nt, 1024);
     L->G = off;       off = align_up(off + g_elem_bytes * static_cast<size_t>(T_chunk) * block_v, 1024);
     L->acc = off;     off = align_up(off + 4 * static_cast<size_t>(T_chunk) * d, 1024);
+    // exact one-hot terms (bf16 path): per-token rounding residue, sorted (target, token) keys, split-run partial sums
+    L->delta = off;   off = align_up(off + 4 * T_chunk, 1024);
+    L->keys = off;    off = align_up(off + 8 * T_chunk, 1024);
+    const size_t segs = (static_cast<size_t>(T_chunk < SORT_MAX ? T_chunk : SORT_MAX) + FIX_SEG - 1) / FIX_SEG;
+    L->partials = off; off = align_up(off + 4 * segs * 2 * static_cast<size_t>(d), 1024);
     L->total = off;
     return true;
 }
@@ -380,6 +395,8 @@ cudaError_t fold_meeting(const FoldCtx& c, int x_row0, int rows, int w_row0, int
 struct GradCtx {
     CUtensorMap tmX_k, tmW_k, tmW_khalf, tmG_st, tmG_k, tmW_mn, tmG_mn, tmX_mn, tmW_mn2, tmX_mn2;
     int* status; float* inv_n; __nv_bfloat16* G;
+    const __nv_bfloat16* X;                 // first row of the X map
+    float* delta; unsigned long long* keys; float* partials;   // exact one-hot terms (see vp_ce_fixup.cuh)
     int g_rows, g_ld;                       // rows and row pitch (elements) of the residual strip in the workspace
     int bn, pmask, ignore_index, V;
     int64_t d;
@@ -389,6 +406,7 @@ struct GradCtx {
 bool make_grad_ctx(GradCtx* c, const void* X, int64_t x_rows, const void* W, int64_t w_rows, int64_t d,
                    __nv_bfloat16* G, int64_t g_rows, int64_t g_ld) {
     c->d = d; c->G = G; c->g_rows = static_cast<int>(g_rows); c->g_ld = static_cast<int>(g_ld);
+    c->X = static_cast<const __nv_bfloat16*>(X);
     c->bn = pick_bn(d);
     c->pmask = pair_mask();
     c->pair_ok = (c->bn == 256) && (d % 64 == 0);
@@ -417,13 +435,27 @@ enum { PHASE_RESIDUAL = VPCE_PHASE_RESIDUAL, PHASE_INPUT_GRAD = VPCE_PHASE_INPUT
 //   input grad   acc (+)= G W_q   (fp32 [rows, d], pitch d; first: overwrite; last: write bf16 dX instead)
 //   weight grad  dW_q (+)= G^T X  (fp32 [cols, d])
 // labels / lse / dloss / acc / dX point at the batch's first token, dW_q at the shard's first row.
+// The range of vocabulary ids whose exact one-hot terms a meeting adds after its GEMMs (nv == 0: none), with the rows
+// of the weight and of the weight gradient that belong to id v0.
+struct FixRange { int v0, nv; const __nv_bfloat16* W_v0; float* dW_v0; bool sort_now; };
+
+cudaError_t sort_targets(const GradCtx& c, const int32_t* labels, int rows, cudaStream_t st) {
+    const int subs = (rows + SORT_MAX - 1) / SORT_MAX;
+    vpce_sort_targets_kernel<<<subs * (SORT_MAX / RANK_TOKENS), RANK_TOKENS * RANK_PARTS, 0, st>>>(labels, rows, c.ignore_index,
+                                                                                                c.V, c.keys);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
 cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int w_row0, int cols, int v_lo,
                          const int32_t* labels, const float* lse, const float* dloss, bool first, bool last, float* acc,
-                         __nv_bfloat16* dX, float* dW_q, bool accumulate_dW, CounterPool& counters, cudaStream_t st) {
+                         __nv_bfloat16* dX, float* dW_q, bool accumulate_dW, const FixRange& fix, CounterPool& counters,
+                         cudaStream_t st) {
     const int strip_tiles_n = (cols + BN_VOCAB - 1) / BN_VOCAB;
     const int m_tiles = (rows + BM - 1) / BM;
     const int d = static_cast<int>(c.d);
     cudaError_t e = cudaSuccess;
+    if ((phases & PHASE_RESIDUAL) && fix.sort_now && (e = sort_targets(c, labels, rows, st)) != cudaSuccess) return e;
     if (phases & PHASE_RESIDUAL) {
         GemmParams p{};
         p.m_tiles = m_tiles;
@@ -436,6 +468,7 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         p.labels = labels; p.lse = lse; p.dloss = dloss;
         p.inv_n_valid = c.inv_n; p.ignore_index = c.ignore_index; p.V = c.V;
         p.G = c.G; p.g_ld = c.g_ld; p.g_rows = c.g_rows;
+        p.delta = c.delta;
         p.status = c.status;
         apply_tuning(p, EPI_RESID);
         p.tile_counter = counters.take();
@@ -469,10 +502,11 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         if ((c.pmask & 2) && c.pair_ok && ph.m_tiles >= 2) e = launch_pair<256, false, true, EPI_DH>(c.tmG_k, c.tmW_mn2, tmAcc, ph, st);
         else e = launch_grad<false, true, EPI_DH>(c.bn, c.tmG_k, c.tmW_mn, tmAcc, ph, st);
         if (e != cudaSuccess) return e;
-        if (last && dX) {
-            const long n8 = static_cast<long>(rows) * d / 8;
-            const long blocks = (n8 + 255) / 256;
-            vpce_acc_to_bf16_kernel<<<static_cast<unsigned>(blocks < 148 * 8 ? blocks : 148 * 8), 256, 0, st>>>(acc, dX, n8);
+        // one pass over the accumulator: dX[n, :] += delta_n W[t_n, :] for the targets in the fix range and, after
+        // the batch's last meeting, the rounding to the bf16 output
+        if (fix.nv > 0 || (last && dX)) {
+            vpce_finish_dx_kernel<<<rows, 128, 0, st>>>(acc, last ? dX : nullptr, fix.nv > 0 ? fix.W_v0 : nullptr, labels,
+                                                       c.delta, d, fix.v0, fix.nv, c.ignore_index);
             g_launches.fetch_add(1, std::memory_order_relaxed);
             if ((e = cudaGetLastError()) != cudaSuccess) return e;
         }
@@ -498,6 +532,18 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         if ((c.pmask & 4) && c.pair_ok && pw.m_tiles >= 2) e = launch_pair<256, true, true, EPI_DW>(c.tmG_mn, c.tmX_mn2, tmDW, pw, st);
         else e = launch_grad<true, true, EPI_DW>(c.bn, c.tmG_mn, c.tmX_mn, tmDW, pw, st);
         if (e != cudaSuccess) return e;
+        if (fix.nv > 0) {                                     // dW[t_n, :] += delta_n X[n, :] for targets in the range
+            const int col_blocks = (d + 255) / 256;
+            for (int r0 = 0; r0 < rows; r0 += SORT_MAX) {     // sub-chunks one after the other: a target may recur
+                const int n_sub = rows - r0 < SORT_MAX ? rows - r0 : SORT_MAX;
+                dim3 grid((n_sub + FIX_SEG - 1) / FIX_SEG, col_blocks);
+                vpce_onehot_dw_kernel<<<grid, 256, 0, st>>>(c.keys + r0, n_sub, c.X + static_cast<size_t>(x_row0) * d,
+                                                            c.delta, d, fix.v0, fix.nv, fix.dW_v0, c.partials);
+                vpce_onehot_dw_combine_kernel<<<grid, 256, 0, st>>>(c.keys + r0, n_sub, d, fix.v0, fix.nv, fix.dW_v0, c.partials);
+                g_launches.fetch_add(2, std::memory_order_relaxed);
+                if ((e = cudaGetLastError()) != cudaSuccess) return e;
+            }
+        }
     }
     return cudaSuccess;
 }
@@ -572,6 +618,9 @@ vpce_status backward_impl(const void* H, const void* W, const int32_t* labels, c
     if (!make_grad_ctx(&c, H, T, W, V, d, reinterpret_cast<__nv_bfloat16*>(ws + L.G), T_chunk, block_v)) return VPCE_CUDA_ERROR;
     c.status = reinterpret_cast<int*>(ws + L.status);
     c.inv_n = reinterpret_cast<float*>(ws + L.scalars);
+    c.delta = reinterpret_cast<float*>(ws + L.delta);
+    c.keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
+    c.partials = reinterpret_cast<float*>(ws + L.partials);
     c.ignore_index = ignore_index; c.V = static_cast<int>(V);
     float* acc = reinterpret_cast<float*>(ws + L.acc);
 
@@ -595,10 +644,13 @@ vpce_status backward_impl(const void* H, const void* W, const int32_t* labels, c
             const int64_t q = ((cg - i) % P + P) % P;
             const int64_t v_lo = q * block_v;
             const int cols = static_cast<int>((V - v_lo) < block_v ? (V - v_lo) : block_v);
+            // the chunk's tokens are sorted by target before its first meeting; after its last one the exact one-hot
+            // terms of ALL shards are added in one go (every token's residue is on record by then)
+            FixRange fix{0, i == P - 1 ? static_cast<int>(V) : 0, static_cast<const __nv_bfloat16*>(W), dW, i == 0};
             if (grad_meeting(c, phases, static_cast<int>(tok0), rows, static_cast<int>(v_lo), cols, static_cast<int>(v_lo),
                              labels + tok0, lse + tok0, dloss ? dloss + tok0 : nullptr, i == 0, i == P - 1, acc,
                              dH ? static_cast<__nv_bfloat16*>(dH) + tok0 * d : nullptr, dW ? dW + v_lo * d : nullptr,
-                             (accumulate_dW != 0) || (ch > 0), counters, st) != cudaSuccess)
+                             (accumulate_dW != 0) || (ch > 0), fix, counters, st) != cudaSuccess)
                 return VPCE_CUDA_ERROR;
         }
     }
@@ -711,6 +763,9 @@ vpce_status vp_ce_meeting_backward(const void* X, const void* W_shard, const int
         return VPCE_CUDA_ERROR;
     c.status = reinterpret_cast<int*>(ws + L.status);
     c.inv_n = reinterpret_cast<float*>(ws + L.scalars);
+    c.delta = reinterpret_cast<float*>(ws + L.delta);
+    c.keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
+    c.partials = reinterpret_cast<float*>(ws + L.partials);
     c.ignore_index = ignore_index; c.V = static_cast<int>(V);
     if (first && (phases & PHASE_RESIDUAL)) {
         vpce_clear_status_kernel<<<1, 32, 0, st>>>(c.status);
@@ -719,9 +774,13 @@ vpce_status vp_ce_meeting_backward(const void* X, const void* W_shard, const int
     CounterPool counters(reinterpret_cast<int*>(ws + L.counters), st);
     // a batch whose only meeting this is (first and last) needs no travelling accumulator: the workspace's own serves
     float* acc = dX_acc ? dX_acc : reinterpret_cast<float*>(ws + L.acc);
+    // every meeting sorts the batch it is handed (it may be another batch each round) and adds the exact one-hot
+    // terms of the targets that lie in its own shard
+    FixRange fix{static_cast<int>(v_lo), static_cast<int>(shard_rows), static_cast<const __nv_bfloat16*>(W_shard), dW_shard,
+                 true};
     if (grad_meeting(c, phases, 0, static_cast<int>(N), 0, static_cast<int>(shard_rows), static_cast<int>(v_lo), targets, lse,
                      dloss, first != 0, last != 0, acc, static_cast<__nv_bfloat16*>(dX), dW_shard, accumulate_dW != 0,
-                     counters, st) != cudaSuccess)
+                     fix, counters, st) != cudaSuccess)
         return VPCE_CUDA_ERROR;
     return counters.failed ? VPCE_CUDA_ERROR : VPCE_OK;
 }

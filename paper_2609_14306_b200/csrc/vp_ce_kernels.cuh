@@ -45,6 +45,7 @@ struct GemmParams {
     float* ylab;                           // [part_ld] target logit
     int part_ld;
     __nv_bfloat16* G;                      // [T_chunk][g_ld]
+    float* delta;                          // [T_chunk] or null: exact minus bf16-rounded value of each token's target entry of G
     int g_ld;
     int g_rows;                            // rows of the G workspace (T_chunk)
     // DH / DW: the fp32 output is described by the launch's third tensor map (boxes of 32 columns x 32 rows)
@@ -174,6 +175,13 @@ __device__ __forceinline__ void epilogue_resid(const GemmParams& p, const CUtens
                 float g = dl * ex2f(fmaf(v[j], LOG2E, -lseL));
                 if (j == jj) g -= dl;
                 v[j] = (j < nvalid) ? g : 0.f;
+            }
+            if (static_cast<unsigned>(jj) < 32u && jj < nvalid && p.delta) {
+                // what bf16 rounding takes from this token's one-hot entry; the fix-up kernels add it back exactly
+                float gx = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) if (j == jj) gx = v[j];
+                p.delta[grow] = gx - __bfloat162float(__float2bfloat16_rn(gx));
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -879,19 +887,6 @@ __global__ void vpce_mean_loss_kernel(const float* __restrict__ loss, const int3
     if (threadIdx.x == 0) {
         *mean_out = cnts[0] > 0 ? static_cast<float>(sums[0] / cnts[0]) : 0.f;
         *n_valid_out = cnts[0];
-    }
-}
-
-// Rounds the finished fp32 input-gradient accumulator of a chunk to the bf16 output (once per chunk).
-__global__ void vpce_acc_to_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ out, long n8) {
-    const long stride = static_cast<long>(gridDim.x) * blockDim.x;
-    for (long i = static_cast<long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += stride) {
-        const float4 a = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i);
-        const float4 b = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i + 1);
-        uint4 o;
-        o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
-        o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
-        reinterpret_cast<uint4*>(out)[i] = o;
     }
 }
 

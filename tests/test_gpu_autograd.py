@@ -87,5 +87,7 @@ def test_autograd_second_backward_and_frozen_weight():
     n0 = vp.vp_ce_launch_count()
     vp.vocab_proj_cross_entropy_mean(H, W, lab, block_v=w.block_v, T_chunk=w.T_chunk).backward()
     both = vp.vp_ce_launch_count() - n0
-    assert both == launches_frozen + meetings                     # the weight-gradient GEMM of every (chunk, shard)
-    assert both == launches_weight_only + meetings + chunks       # the input-gradient GEMMs + one rounding pass per chunk
+    # without dW: no weight-gradient GEMM per (chunk, shard) and no one-hot scatter (two launches) per chunk
+    assert both == launches_frozen + meetings + 2 * chunks
+    # without dH: no input-gradient GEMM per (chunk, shard) and no finishing pass over the accumulator per chunk
+    assert both == launches_weight_only + meetings + chunks

@@ -100,7 +100,7 @@ def check_call(w, call, W_bits, W64, labels_stream, n_valid_total, T_chunk, W_de
     assert not run.dH[torch.from_numpy(np.nonzero(labels == IGNORE_INDEX)[0]).cuda()].any()
     # invariant: every residual row sums to zero, so the column sums of dW vanish (up to bf16 rounding of G)
     colsum = run.dW.double().sum(0)
-    assert float(colsum.norm() / run.dW.double().norm()) < 5e-3
+    assert float(colsum.norm() / run.dW.double().norm()) < 5e-4
     mean_gpu, n_valid = run.mean()
     valid = labels != IGNORE_INDEX
     assert n_valid == int(valid.sum())
