@@ -86,6 +86,9 @@ vpce_status vp_ce_forward(const void* H, const void* W, const int32_t* labels,
  * added to otherwise (fp32 accumulation across calls of a streamed context).
  * Either dH or dW (not both) may be NULL: that gradient and its contraction are skipped
  * (a frozen projection weight, or an input that needs no gradient).
+ * The residual strip is staged as bf16, but the target entry of every token's row is applied
+ * exactly: what rounding took from it is added back to dH and dW in fp32, in a fixed order, so
+ * results are bitwise reproducible and the one-hot part of the gradients carries no rounding bias.
  */
 vpce_status vp_ce_backward(const void* H, const void* W, const int32_t* labels, const float* lse,
                            const float* dloss, void* dH, float* dW,

@@ -330,3 +330,33 @@ def test_profile_hooks_count_launches_per_kernel_kind():
         assert n == meetings and ms > 0.0
     assert vp.vp_ce_launch_count() - n0 >= 4 * meetings
     assert all(n == 0 for _, n in vp.vp_ce_profile_collect().values())     # collected entries are forgotten
+
+
+def test_forward_and_backward_replay_from_a_cuda_graph():
+    """The calls only enqueue work on the caller's stream (no host synchronisation, no allocation), so a forward +
+    backward pair can be captured once and replayed: the replays reproduce the directly launched results bit for bit."""
+    w = custom_workload("graph", T=512, d=256, V=2048, block_v=512, T_chunk=256, w_std=0.0625, labels="zipf",
+                        ignore_frac=0.05, seed=71)
+    b = make_batch(w)
+    direct = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk, 2).forward().backward()
+    r = DeviceRun(b.H_bits, b.W_bits, b.labels, w.block_v, w.T_chunk, 2)
+    r.dH = torch.zeros(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+    r.dW = torch.zeros(w.V, w.d, dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                      # warm-up outside the capture (module load, function attributes)
+        vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, 2, r.ws)
+        vp.vp_ce_backward(r.H, r.W, r.labels, r.lse, None, r.dH, r.dW, w.block_v, IGNORE_INDEX, w.T_chunk, 2, False, r.ws)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        vp.vp_ce_forward(r.H, r.W, r.labels, w.block_v, IGNORE_INDEX, r.loss, r.lse, w.T_chunk, 2, r.ws)
+        vp.vp_ce_backward(r.H, r.W, r.labels, r.lse, None, r.dH, r.dW, w.block_v, IGNORE_INDEX, w.T_chunk, 2, False, r.ws)
+    for _ in range(2):
+        r.loss.fill_(float("nan")); r.lse.fill_(float("nan")); r.dH.zero_(); r.dW.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert vp.vp_ce_device_status(r.ws) == 0
+        assert torch.equal(r.lse, direct.lse) and torch.equal(r.loss, direct.loss)
+        assert torch.equal(r.dH.view(torch.int16), direct.dH.view(torch.int16)) and torch.equal(r.dW, direct.dW)
