@@ -42,6 +42,7 @@ def test_config2_mid():
     (512, 2880, 2048, 512, 256),    # d = 2880 selects the 192-column gradient tile
     (384, 512, 5000, 1024, 384),    # T_chunk of three tiles, 5 shards, last one ragged
     (200, 64, 600, 512, 1024),      # T_chunk larger than the batch: one short chunk
+    (16640, 64, 1000, 512, 16640),  # a chunk of more than 16384 tokens: the one-hot scatter sorts it in two sub-chunks
 ])
 def test_ragged_shapes(T, d, V, block_v, T_chunk):
     w = custom_workload(f"r{T}x{d}x{V}", T=T, d=d, V=V, block_v=block_v, T_chunk=T_chunk,
