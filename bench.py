@@ -631,13 +631,15 @@ def main():
     out = measure(ctx, w, args.dtype, args.steps, args.warmup, t_chunk=args.t_chunk, with_e2e=not args.no_e2e,
                   with_cpu_baseline=not args.no_cpu_baseline, with_yardstick=not args.no_yardstick, prof_on=prof_on)
     # The default run also measures, in the same process and through the same code, the OTHER configuration the
-    # throughput target is stated on (config 4) and the paper's own benchmark shape in the paper's precision
-    # (FP32 inputs on TF32 tensor cores): fewer steps, no CPU leg.  One GPU only, so that a scaling run stays short.
+    # throughput target is stated on (config 4), the long-context stream (config 5: 64 calls per step, same workspace as
+    # config 3), the paper's own benchmark shape in the paper's precision (FP32 inputs on TF32 tensor cores) and the
+    # streamed AdamW: fewer steps, no CPU leg.  One GPU only, so that a scaling run stays short.
     if ctx.rank == 0 and ctx.world == 1 and not args.no_also and args.workload == "moe120b" and args.dtype == "bf16":
         k = max(3, min(args.steps, 5))
         out["also"] = [
             measure(ctx, WORKLOADS["moe667b"], "bf16", k, 3, with_e2e=not args.no_e2e, with_cpu_baseline=False,
                     with_yardstick=not args.no_yardstick, prof_on=prof_on),
+            measure(ctx, WORKLOADS["longctx"], "bf16", 2, 3, with_e2e=False, with_cpu_baseline=False, prof_on=prof_on),
             measure(ctx, PROFILE_WORKLOADS["papershape"], "tf32", 3, 3, with_e2e=False, with_cpu_baseline=False,
                     prof_on=prof_on),
             measure_adamw(ctx, n_params=1 << 28, bucket=1 << 25, slots=2, steps=3, warmup=2),
