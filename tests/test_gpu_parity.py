@@ -361,3 +361,30 @@ def test_forward_and_backward_replay_from_a_cuda_graph():
         assert vp.vp_ce_device_status(r.ws) == 0
         assert torch.equal(r.lse, direct.lse) and torch.equal(r.loss, direct.loss)
         assert torch.equal(r.dH.view(torch.int16), direct.dH.view(torch.int16)) and torch.equal(r.dW, direct.dW)
+
+
+@pytest.mark.parametrize("pattern", ["one_target", "two_targets_offset", "blocks_of_65"])
+def test_long_runs_of_equal_targets_in_the_one_hot_scatter(pattern):
+    """Targets that repeat over many consecutive sorted positions: a run then spans several 64-position segments of the
+    scatter (partial sums combined in segment order), starts in the middle of a segment, or ends exactly at a boundary."""
+    w = custom_workload("runs", T=1024, d=320, V=768, block_v=512, T_chunk=1024, w_std=0.3, labels="uniform",
+                        ignore_frac=0.0, seed=81)
+    b = make_batch(w)
+    lab = b.labels.copy()
+    if pattern == "one_target":
+        lab[:] = 7
+        lab[::50] = IGNORE_INDEX
+    elif pattern == "two_targets_offset":
+        lab[:] = 600                       # lives in the second shard
+        lab[:37] = 3                       # 37 tokens of one target, then a run that starts mid-segment
+    else:
+        lab[:] = (np.arange(w.T) // 65) % w.V      # runs of 65: every run crosses a segment boundary somewhere
+    H64, W64 = bf16_bits_to_f64(b.H_bits), bf16_bits_to_f64(b.W_bits)
+    dl = (0.5 + np.random.default_rng(5).random(w.T)).astype(np.float32) / w.T
+    ref = orc.forward_backward(H64, W64, lab, dl.astype(np.float64))
+    runs = [DeviceRun(b.H_bits, b.W_bits, lab, w.block_v, w.T_chunk).forward().backward(dloss=dl) for _ in range(2)]
+    r = runs[0]
+    assert r.fwd_status == 0 and r.bwd_status == 0
+    assert torch.equal(runs[0].dW, runs[1].dW) and torch.equal(runs[0].dH.view(torch.int16), runs[1].dH.view(torch.int16))
+    e = check_against_oracle(r, ref, H64, W64, lab, dl.astype(np.float64), pattern)
+    assert e["dW"] <= 1e-3, e                          # with exact one-hot terms dW is far inside the 1e-2 gate
