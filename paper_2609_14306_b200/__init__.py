@@ -45,6 +45,9 @@ def __getattr__(name):
     if name in ("vocab_proj_cross_entropy", "vocab_proj_cross_entropy_mean"):
         from . import autograd as _ag
         return getattr(_ag, name)
+    if name == "HostStepPipeline":
+        from . import host_pipeline as _hp
+        return _hp.HostStepPipeline
     if name in ("RingDTP", "DistTransport", "CudaMeetings", "choose_schedule", "shard_interval"):
         from . import ring as _ring
         return getattr(_ring, name)

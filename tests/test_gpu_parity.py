@@ -388,3 +388,32 @@ def test_long_runs_of_equal_targets_in_the_one_hot_scatter(pattern):
     assert torch.equal(runs[0].dW, runs[1].dW) and torch.equal(runs[0].dH.view(torch.int16), runs[1].dH.view(torch.int16))
     e = check_against_oracle(r, ref, H64, W64, lab, dl.astype(np.float64), pattern)
     assert e["dW"] <= 1e-3, e                          # with exact one-hot terms dW is far inside the 1e-2 gate
+
+
+def test_host_step_pipeline_overlaps_copies_and_matches_oracle():
+    """HostStepPipeline: several steps in flight on two staging slots; every step's host outputs match the oracle."""
+    w = custom_workload("pipe", T=512, d=256, V=2000, block_v=1024, T_chunk=256, w_std=0.0625, labels="zipf",
+                        ignore_frac=0.1, seed=91)
+    Wb = make_batch(w).W_bits
+    Wd = torch.from_numpy(Wb.view(np.int16)).cuda().view(torch.bfloat16)
+    W64 = bf16_bits_to_f64(Wb)
+    dW = torch.full((w.V, w.d), float("nan"), device="cuda")
+    pipe = vp.HostStepPipeline(Wd, dW, w.T, w.d, w.block_v, w.T_chunk, IGNORE_INDEX, depth=2)
+    steps = []
+    for i in range(5):                                    # distinct data per step, more steps than slots
+        wi = custom_workload("pipe", T=w.T, d=w.d, V=w.V, block_v=w.block_v, T_chunk=w.T_chunk, w_std=0.0625, labels="zipf",
+                             ignore_frac=0.1, seed=91 + i)
+        bi = make_batch(wi, W_bits=Wb)
+        Hh = torch.from_numpy(bi.H_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+        lh = torch.from_numpy(bi.labels).pin_memory()
+        loss_h = torch.full((w.T,), float("nan")).pin_memory()
+        dH_h = torch.zeros(w.T, w.d, dtype=torch.bfloat16).pin_memory()
+        pipe.submit(Hh, lh, loss_h, dH_h)
+        steps.append((bi, Hh, lh, loss_h, dH_h))
+    pipe.wait()
+    assert pipe.device_status() == 0
+    for bi, _, _, loss_h, dH_h in steps:
+        ref = orc.forward_backward(bf16_bits_to_f64(bi.H_bits), W64, bi.labels)
+        assert np.abs(loss_h.numpy().astype(np.float64) - ref["loss"]).max() <= TOL_TOKEN
+        assert relF(dH_h.float().numpy().astype(np.float64), ref["dH"]) <= TOL_GRAD
+    assert relF(dW.cpu().numpy().astype(np.float64), ref["dW"]) <= TOL_GRAD      # the last step's (dW is overwritten)
