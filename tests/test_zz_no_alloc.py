@@ -72,17 +72,18 @@ def test_static_scratch_call_takes_no_device_memory():
     loss, lse, _ = _static_forward(w, H, W, lab, base=0)          # first call: module load, address look-up
     vp.vp_ce_profile_enable(True)                                  # the event-recording path must not be taken either
     try:
-        torch.cuda.synchronize()
-        free0, _ = torch.cuda.mem_get_info()
-        alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
         status = torch.zeros(1, dtype=torch.int32, device="cuda")      # allocated before the measured window
+        # what earlier tests left behind (tensors, a captured graph's pool) is released now, not inside the window
+        import gc
+        gc.collect()
+        torch.cuda.synchronize()
         free0, _ = torch.cuda.mem_get_info()
         alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
         vp.vp_ce_forward_static(H, W, lab, w.block_v, IGNORE_INDEX, loss, lse, w.T_chunk, 0, status)
         torch.cuda.synchronize()
         free1, _ = torch.cuda.mem_get_info()
         assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
-        assert free1 == free0, (free0, free1)                      # the driver handed out nothing either
+        assert free1 >= free0, (free0, free1)                      # the driver handed out nothing either
     finally:
         vp.vp_ce_profile_enable(False)
     assert all(n == 0 for _, n in vp.vp_ce_profile_collect().values())
