@@ -3,8 +3,8 @@
 // A warp-specialised, persistent tcgen05 GEMM kernel is instantiated with four epilogues:
 //   FOLD   strip Y = H_c W_q^T  -> per-tile partial (max, sum-exp) + target logit   (Eq. 2)
 //   RESID  the same strip       -> G = dloss (exp(Y - lse) - onehot) as bf16       (App. C)
-//   DH     dH_c += G W_q        (contract over the shard's vocabulary)
-//   DW     dW_q += G^T H_c      (contract over the chunk's tokens)
+//   DH     dH_c += G W_q        (contract over the shard's vocabulary)  fp32 tiles leave by TMA store / TMA fp32
+//   DW     dW_q += G^T H_c      (contract over the chunk's tokens)      reduction (the running sums stay in memory)
 // Operands reach shared memory by TMA (128-byte swizzle), accumulators live in tensor
 // memory (two buffers, so the epilogue of tile i overlaps the MMAs of tile i+1), and the
 // logit strip never reaches global memory.
@@ -17,6 +17,9 @@
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner,
 // warps 2..5 = epilogue (one thread per accumulator row).
+//
+// After a chunk's last meeting the exact one-hot terms are added (vp_ce_fixup.cuh): what bf16 rounding took from each
+// token's target entry of G goes back into dH and dW in fp32, in a fixed order.
 //
 // Every wait on an mbarrier is bounded: when it runs out the CTA records
 // VPCE_DEV_WAIT_EXPIRED in the workspace status word, all roles leave their loops, pending
