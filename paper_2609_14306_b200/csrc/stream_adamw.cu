@@ -190,31 +190,43 @@ int osadamw_step(osadamw_ctx* c, float* master, float* m, float* v, const float*
     for (int64_t b = 0; b < n_buckets; ++b) {
         const int64_t a0 = bucket_offsets ? bucket_offsets[b] : b * c->bucket;
         const int64_t a1 = bucket_offsets ? bucket_offsets[b + 1] : (a0 + c->bucket < n ? a0 + c->bucket : n);
-        const size_t len = static_cast<size_t>(a1 - a0), bytes = len * sizeof(float);
+        const size_t len = static_cast<size_t>(a1 - a0);
         const int k = static_cast<int>(b % c->slots);
         float* sp = c->staging + static_cast<size_t>(k) * 4 * sf;
         float *sm = sp + sf, *sv = sp + 2 * sf, *sg = sp + 3 * sf;
         // (i) a slot is free again once its write-back has completed (Algorithm 4: "wait for a free staging slot")
         if (c->used[k] && cudaStreamWaitEvent(c->s_in, c->written[k], 0) != cudaSuccess) return VPCE_CUDA_ERROR;
         c->used[k] = 1;
-        if (cudaMemcpyAsync(sp, master + a0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
-            cudaMemcpyAsync(sm, m + a0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
-            cudaMemcpyAsync(sv, v + a0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
-            cudaMemcpyAsync(sg, grad + a0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
-            cudaEventRecord(c->loaded[k], c->s_in) != cudaSuccess)
-            return VPCE_CUDA_ERROR;
-        // (ii) fused update + bf16 refresh
-        if (cudaStreamWaitEvent(c->s_upd, c->loaded[k], 0) != cudaSuccess ||
-            launch_update(sp, sm, sv, sg, static_cast<__nv_bfloat16*>(w_bf16) + a0, static_cast<long>(len), sc, c->s_upd) != cudaSuccess ||
-            cudaEventRecord(c->updated[k], c->s_upd) != cudaSuccess)
-            return VPCE_CUDA_ERROR;
-        // (iii) write the fp32 state back
-        if (cudaStreamWaitEvent(c->s_out, c->updated[k], 0) != cudaSuccess ||
-            cudaMemcpyAsync(master + a0, sp, bytes, cudaMemcpyDeviceToHost, c->s_out) != cudaSuccess ||
-            cudaMemcpyAsync(m + a0, sm, bytes, cudaMemcpyDeviceToHost, c->s_out) != cudaSuccess ||
-            cudaMemcpyAsync(v + a0, sv, bytes, cudaMemcpyDeviceToHost, c->s_out) != cudaSuccess ||
-            cudaEventRecord(c->written[k], c->s_out) != cudaSuccess)
-            return VPCE_CUDA_ERROR;
+        // Inside a bucket the three stages run piece by piece (up to 8 pieces of at least 4 Mi parameters), so the update
+        // and the write-back of a large bucket start when its first piece has arrived, not when all of it has: filling
+        // and draining the pipeline then costs a piece, not a bucket.  An event may be recorded again while an earlier
+        // wait on it is pending: a wait refers to the record that was current when the wait was enqueued.
+        size_t piece = (len + 7) / 8;
+        if (piece < (4u << 20)) piece = 4u << 20;
+        piece = (piece + 3) / 4 * 4;
+        for (size_t o = 0; o < len; o += piece) {
+            const size_t l = len - o < piece ? len - o : piece, bytes = l * sizeof(float);
+            const int64_t g0 = a0 + static_cast<int64_t>(o);
+            if (cudaMemcpyAsync(sp + o, master + g0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
+                cudaMemcpyAsync(sm + o, m + g0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
+                cudaMemcpyAsync(sv + o, v + g0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
+                cudaMemcpyAsync(sg + o, grad + g0, bytes, cudaMemcpyHostToDevice, c->s_in) != cudaSuccess ||
+                cudaEventRecord(c->loaded[k], c->s_in) != cudaSuccess)
+                return VPCE_CUDA_ERROR;
+            // (ii) fused update + bf16 refresh
+            if (cudaStreamWaitEvent(c->s_upd, c->loaded[k], 0) != cudaSuccess ||
+                launch_update(sp + o, sm + o, sv + o, sg + o, static_cast<__nv_bfloat16*>(w_bf16) + g0, static_cast<long>(l), sc,
+                              c->s_upd) != cudaSuccess ||
+                cudaEventRecord(c->updated[k], c->s_upd) != cudaSuccess)
+                return VPCE_CUDA_ERROR;
+            // (iii) write the fp32 state back
+            if (cudaStreamWaitEvent(c->s_out, c->updated[k], 0) != cudaSuccess ||
+                cudaMemcpyAsync(master + g0, sp + o, bytes, cudaMemcpyDeviceToHost, c->s_out) != cudaSuccess ||
+                cudaMemcpyAsync(m + g0, sm + o, bytes, cudaMemcpyDeviceToHost, c->s_out) != cudaSuccess ||
+                cudaMemcpyAsync(v + g0, sv + o, bytes, cudaMemcpyDeviceToHost, c->s_out) != cudaSuccess ||
+                cudaEventRecord(c->written[k], c->s_out) != cudaSuccess)
+                return VPCE_CUDA_ERROR;
+        }
     }
     // later work on the caller's stream sees the refreshed working weight
     if (cudaEventRecord(c->ev_last_update, c->s_upd) != cudaSuccess ||
