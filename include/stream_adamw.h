@@ -9,7 +9,9 @@
  * the AdamW update in fp32 and refreshes the bf16 working weight, (iii) copy of the updated fp32 state back to
  * the host.  A slot is taken again only after its write-back has finished.  The three stages of different
  * buckets overlap, so a step costs about (number of buckets) x max(copy in, update, copy out)   (Eq. 4), and the
- * staging memory is slots x bucket_params x 16 bytes.
+ * staging memory is slots x bucket_params x 16 bytes.  Inside a bucket the stages run piece by piece (up to 8 pieces
+ * of at least 4 Mi parameters), so the update and write-back of a large bucket begin when its first piece has
+ * arrived; the results do not depend on the bucketing (the rule is elementwise).
  *
  * The update of one parameter with gradient g at step t = 1, 2, ... (decoupled weight decay; the appendix says
  * the fused kernel keeps the reference implementation's bias correction, weight decay and update order):
