@@ -91,3 +91,15 @@ def test_autograd_second_backward_and_frozen_weight():
     assert both == launches_frozen + meetings + 2 * chunks
     # without dH: no input-gradient GEMM per (chunk, shard) and no finishing pass over the accumulator per chunk
     assert both == launches_weight_only + meetings + chunks
+
+
+def test_autograd_empty_batch():
+    d, V = 64, 512
+    H = torch.empty(0, d, dtype=torch.bfloat16, device="cuda", requires_grad=True)
+    W = (torch.randn(V, d, device="cuda") * 0.1).to(torch.bfloat16).requires_grad_(True)
+    lab = torch.empty(0, dtype=torch.int64, device="cuda")
+    loss = vp.vocab_proj_cross_entropy_mean(H, W, lab, block_v=256)
+    assert float(loss.detach()) == 0.0                         # no valid token: mean 0 (the documented rule)
+    loss.backward()
+    assert H.grad.shape == (0, d)
+    assert W.grad is not None and not W.grad.any()             # an empty batch contributes nothing
