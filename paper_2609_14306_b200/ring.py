@@ -110,6 +110,21 @@ class CudaMeetings:
     def forward_meeting(self, X, W, t, v_lo, V, ignore_index, state, first, last, loss, lse, ws) -> None:
         _b.vp_ce_meeting_forward(X, W, t, v_lo, V, ignore_index, state, first, last, loss, lse, ws)
 
+    def count_valid(self, t, V, ignore_index) -> int:
+        """Number of tokens whose target is neither ignore_index nor outside [0, V) (vp_ce_mean_loss's count)."""
+        zeros = torch.zeros(t.numel(), dtype=torch.float32, device=t.device)
+        mean = torch.empty(1, dtype=torch.float32, device=t.device)
+        n = torch.empty(1, dtype=torch.int32, device=t.device)
+        _b.vp_ce_mean_loss(zeros, t, V, ignore_index, mean, n)
+        return int(n.item())
+
+    def mean_dloss(self, t, V, ignore_index, n_valid_total: int) -> torch.Tensor:
+        """1 / n_valid_total on valid tokens, 0 elsewhere (vp_ce_mean_loss_grad)."""
+        n = torch.tensor([int(n_valid_total)], dtype=torch.int32, device=t.device)
+        out = torch.empty(t.numel(), dtype=torch.float32, device=t.device)
+        _b.vp_ce_mean_loss_grad(t, V, ignore_index, n, None, out)
+        return out
+
     def backward_meeting(self, X, W, t, lse, dloss, v_lo, V, ignore_index, phases, dX_acc, first, last, dX, dW,
                          accumulate_dW, ws) -> None:
         _b.vp_ce_meeting_backward(X, W, t, lse, dloss, v_lo, V, ignore_index, phases, dX_acc, first, last, dX, dW,
@@ -160,11 +175,10 @@ class RingDTP:
 
     def masked_mean_dloss(self, t: torch.Tensor) -> torch.Tensor:
         """Upstream gradient of the mean loss over the valid tokens of ALL ranks' batches: 1 / n_valid_total on
-        valid tokens (one integer all-reduce; the paper's operator itself outputs per-token values)."""
-        valid = (t != self.ignore_index) & (t >= 0) & (t < self.V)
-        total = self.tp.all_sum(int(valid.sum().item()))
-        return torch.where(valid, 1.0 / max(total, 1), 0.0).to(torch.float32) if total else torch.zeros(
-            t.shape, dtype=torch.float32, device=t.device)
+        valid tokens (one integer all-reduce of the local counts; the paper's operator itself outputs per-token
+        values).  The counting and the per-token values come from the meetings object (the CUDA library)."""
+        total = self.tp.all_sum(self.meetings.count_valid(t, self.V, self.ignore_index))
+        return self.meetings.mean_dloss(t, self.V, self.ignore_index, total)
 
     # ---- forward
     def forward(self, X: torch.Tensor, t: torch.Tensor, W_own: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
@@ -255,6 +269,8 @@ class RingDTP:
             Wb[0][W_own.shape[0]:].zero_()
         for b in Db:
             b.zero_()                                     # padding rows stay zero on the wire
+        if accumulate_dW:
+            Db[0][: W_own.shape[0]].copy_(dW_own)         # the travelling gradient starts from what the owner holds
         grad_moving = None
         for i in range(P):
             q = (r - i) % P
@@ -266,18 +282,14 @@ class RingDTP:
             if grad_moving is not None:
                 grad_moving.wait()                        # the partial dW_q of the ranks that met q before this one
             M.backward_meeting(X, Wb[c][: hi - lo], t, lse, dloss, lo, self.V, self.ignore_index, WG, None, i == 0,
-                               i == P - 1, None, Db[c][: hi - lo], i > 0, ws)
+                               i == P - 1, None, Db[c][: hi - lo], i > 0 or accumulate_dW, ws)
             self._note("bwd", i, r, q)
             # the gradient travels with its shard; after the last round this hop brings every dW_q home
             grad_moving = self.tp.exchange([Db[c]], [Db[n]])
             if w_moving is not None:
                 w_moving.wait()
         grad_moving.wait()
-        home = Db[P % 2][: W_own.shape[0]]
-        if accumulate_dW:
-            dW_own.add_(home)
-        else:
-            dW_own.copy_(home)
+        dW_own.copy_(Db[P % 2][: W_own.shape[0]])           # this rank's own shard is home again, complete
         return dX, dW_own
 
     def _backward_move_activations(self, X, t, W_own, lse, dloss, dW_own, accumulate_dW, N):

@@ -61,6 +61,17 @@ class OracleMeetings:
         self.calls.append(("bwd", v_lo, Wn.shape[0], phases, bool(first), bool(last)))
 
 
+    def count_valid(self, t, V, ignore_index):
+        tn = t.numpy()
+        return int(((tn != ignore_index) & (tn >= 0) & (tn < V)).sum())
+
+    def mean_dloss(self, t, V, ignore_index, n_valid_total):
+        tn = t.numpy()
+        valid = (tn != ignore_index) & (tn >= 0) & (tn < V)
+        out = np.where(valid, 1.0 / n_valid_total if n_valid_total else 0.0, 0.0)
+        return torch.from_numpy(out.astype(np.float32))
+
+
 def global_problem(P, N, d, V, seed, ignore_frac=0.1, ignore_index=-100):
     """One seeded problem for a whole group: per-rank batches X_r [N, d], targets, and the full weight."""
     rng = np.random.default_rng(seed)

@@ -22,8 +22,8 @@ class ThreadTransport:
     """Ring of host threads: `exchange` hands finished copies to the next rank's queue; `wait` takes what the
     previous rank handed over and copies it into the receive buffers."""
 
-    def __init__(self, rank, size, queues):
-        self.rank, self.size, self.queues = rank, size, queues
+    def __init__(self, rank, size, queues, shared=None):
+        self.rank, self.size, self.queues, self.shared = rank, size, queues, shared
 
     def exchange(self, send, recv):
         copies = [s.clone() for s in send]
@@ -40,7 +40,12 @@ class ThreadTransport:
         return Handle()
 
     def all_sum(self, value):
-        raise NotImplementedError
+        slots, barrier = self.shared
+        slots[self.rank] = int(value)
+        barrier.wait(timeout=120)
+        total = sum(slots)
+        barrier.wait(timeout=120)                             # nobody overwrites a slot before all have read
+        return total
 
 
 def _problem(P, N, d, V, seed):
@@ -103,6 +108,56 @@ def test_ring_threads_on_one_gpu_match_the_oracle(P, N, d, V, mode):
         dW_all[lo:hi] = dW
         assert len([1 for w_, *_ in log if w_ == "fwd"]) == P and len([1 for w_, *_ in log if w_ == "bwd"]) == P
     assert relF(dW_all, ref["dW"]) <= TOL_GRAD
+
+
+@pytest.mark.parametrize("mode", ["weights", "activations"])
+def test_ring_mean_loss_gradient_and_accumulation_into_an_existing_dW(mode):
+    # the upstream gradient of the group-wide masked mean comes from the library (count + 1/n on valid tokens),
+    # and a second backward with accumulate_dW adds to what dW_own already holds
+    P, N, d, V = 2, 256, 128, 1100
+    Xb, Wb, t = _problem(P, N, d, V, seed=77)
+    t[5] = V + 3                                              # an out-of-range target counts as ignored
+    X64, W64 = bf16_bits_to_f64(Xb), bf16_bits_to_f64(Wb)
+    valid = (t != IGNORE_INDEX) & (t >= 0) & (t < V)
+    dl = np.where(valid, 1.0 / valid.sum(), 0.0)
+    t_ref = np.where(valid, t, IGNORE_INDEX).astype(np.int32)
+    ref = orc.forward_backward(X64, W64, t_ref, dl, IGNORE_INDEX)
+    queues = [queue.Queue() for _ in range(P)]
+    shared = ([0] * P, threading.Barrier(P))
+    out, errors = {}, []
+
+    def rank_main(r):
+        try:
+            lo, hi = ring.shard_interval(r, V, P)
+            Xr = to_dev_bf16(Xb[r * N:(r + 1) * N])
+            Wr = to_dev_bf16(Wb[lo:hi])
+            tr = torch.from_numpy(t[r * N:(r + 1) * N]).cuda()
+            drv = ring.RingDTP(ThreadTransport(r, P, queues, shared), V, d, IGNORE_INDEX, mode=mode)
+            loss, lse = drv.forward(Xr, tr, Wr)
+            dlr = drv.masked_mean_dloss(tr)
+            dX, dW = drv.backward(Xr, tr, Wr, lse, dlr)
+            once = dW.clone()
+            dX2, dW2 = drv.backward(Xr, tr, Wr, lse, dlr, dW_own=dW, accumulate_dW=True)
+            torch.cuda.synchronize()
+            out[r] = (dlr.cpu().numpy(), dX.float().cpu().numpy(), once.cpu().numpy(), dW2.cpu().numpy(),
+                      dX2.float().cpu().numpy())
+        except Exception as exc:
+            errors.append((r, repr(exc)))
+
+    threads = [threading.Thread(target=rank_main, args=(r,)) for r in range(P)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join(timeout=300)
+    assert not errors, errors
+    for r in range(P):
+        dlr, dX, once, twice, dX2 = out[r]
+        sl = slice(r * N, (r + 1) * N)
+        lo, hi = ring.shard_interval(r, V, P)
+        assert np.array_equal(dlr, dl[sl].astype(np.float32))
+        assert relF(dX, ref["dH"][sl]) <= TOL_GRAD and np.array_equal(dX, dX2)
+        assert relF(once, ref["dW"][lo:hi]) <= TOL_GRAD
+        assert relF(twice, 2.0 * ref["dW"][lo:hi]) <= TOL_GRAD
 
 
 def test_meeting_entry_points_reject_bad_arguments():
