@@ -54,6 +54,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
+// A flag in global memory that orders the TMA stores / reductions of one warp before those of another warp (of any
+// CTA): the writer waits for its bulk groups to complete, then publishes; the reader acquires, then issues its own.
+// The proxy fences order the generic-proxy flag accesses against the async-proxy copies on both sides.
+__device__ __forceinline__ void flag_release(int* flag, int value) {
+    asm volatile("fence.proxy.async;" ::: "memory");
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
+}
+// Waits until *flag >= value; gives up (false, abort flag set) after limit_ns or when the CTA has given up already.
+__device__ __forceinline__ bool flag_wait_ge(const int* flag, int value, volatile int* abort_flag, unsigned long long limit_ns) {
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v >= value) {
+            asm volatile("fence.proxy.async;" ::: "memory");
+            return true;
+        }
+        if ((it & 15u) == 15u) {
+            if (*abort_flag) return false;
+            unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
+        }
+        __nanosleep(64);
+    }
+}
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }

@@ -35,7 +35,10 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
+#include <functional>
+#include <map>
 #include <mutex>
+#include <tuple>
 #include <vector>
 
 #include "vp_ce.h"
@@ -250,7 +253,9 @@ cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     const int tiles = ((p.m_tiles + 1) / 2) * p.n_tiles;
     if (tiles <= 0 || p.num_kb <= 0) return cudaSuccess;
     const int max_pairs = num_sms() / 2;
-    const int grid = 2 * (tiles < max_pairs ? tiles : max_pairs);
+    const int n_cut = (EPI == EPI_DH || EPI == EPI_DW) ? std::min(p.n_cut, tiles) : 0;
+    const int entries = tiles + n_cut * (std::max(p.k_split, 1) - 1);          // split tiles count once per part
+    const int grid = 2 * (entries < max_pairs ? entries : max_pairs);
     ProfEntry pe{EPI, nullptr, nullptr};
     bool prof = false;
     {
@@ -269,13 +274,102 @@ cudaError_t launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     return cudaGetLastError();
 }
 
-// How many of the last tiles of a gradient GEMM to run as two 128-column halves: after the whole
-// rounds R = tiles % pairs tiles are left; as halves they finish in about 0.56 tile times instead of
-// one, provided the 2R halves fit into one round (a half costs a little more than half a tile: it
-// re-loads A and uses only half of each B box).
-int pick_n_cut(int pm_tiles, int n_tiles, int pairs) {
-    const int R = pairs > 0 ? (pm_tiles * n_tiles) % pairs : 0;
-    return (R > 0 && 2 * R <= pairs) ? R : 0;
+// The tail of a gradient GEMM's work list.  The pair kernel hands out 256 x 256 tiles greedily; when their number is
+// not a multiple of the number of CTA pairs the last round runs with most pairs idle.  The last n_cut tiles of the list
+// are therefore run as ks parts along K (the parts add into the output in a fixed order, see the kernel).  n_cut and ks
+// come from simulating the greedy hand-out, in units of one k-block of a whole tile: a narrower last n-tile of a row is
+// bound by its operand loads and costs about 7/8 of a whole tile down to an MMA width of half a tile; every part pays
+// for filling the pipeline (TAIL_FILL) and its epilogue, which starts only after the epilogue of the part before it
+// (TAIL_EPI; both constants fitted to measured launch times of the two benchmark geometries).  Part j + 1 is made
+// TAIL_EPI k-blocks longer than part j so that parts that start together finish an epilogue apart.  Decisions are
+// cached per geometry.
+struct SplitChoice { int n_cut, ks, stagger; };
+constexpr int MAX_SPLIT_TILES = 64;            // 8 flags each: half of the counter pool at most
+constexpr double TAIL_FILL = 6.0, TAIL_EPI = 15.0;
+constexpr int TAIL_MIN_PART = 8;               // k-blocks of the shortest part
+
+double simulate_tail(int pm_tiles, int n_tiles, int group_n, double c_last, int n_cut, int ks, int stagger, int num_kb,
+                     int pairs) {
+    const int total = pm_tiles * n_tiles;
+    std::vector<double> heap(pairs, 0.0);       // min-heap of the times at which the pairs become free
+    auto take = [&]() {
+        std::pop_heap(heap.begin(), heap.end(), std::greater<double>());
+        return heap.back();
+    };
+    auto put = [&](double t) {
+        heap.back() = t;
+        std::push_heap(heap.begin(), heap.end(), std::greater<double>());
+    };
+    auto cost = [&](int t) {
+        const int per_group = group_n * pm_tiles;
+        const int g = t / per_group, r = t - g * per_group, n0 = g * group_n;
+        const int gw = std::min(group_n, n_tiles - n0);
+        const int nt = n0 + (r - (r / gw) * gw);
+        return nt == n_tiles - 1 ? c_last : 1.0;
+    };
+    for (int t = 0; t < total - n_cut; ++t) put(take() + num_kb * cost(t));
+    const int base_len = ks > 0 ? (num_kb - stagger * (ks * (ks - 1) / 2)) / ks : num_kb;
+    for (int t = total - n_cut; t < total; ++t) {
+        double prev_done = 0.0;
+        int k0 = 0;
+        for (int j = 0; j < ks; ++j) {
+            const int k1 = j + 1 == ks ? num_kb : k0 + base_len + stagger * j;
+            const double computed = take() + TAIL_FILL + (k1 - k0) * cost(t);
+            prev_done = std::max(computed, prev_done) + TAIL_EPI;
+            put(prev_done);
+            k0 = k1;
+        }
+    }
+    return *std::max_element(heap.begin(), heap.end());
+}
+
+SplitChoice pick_split(int pm_tiles, int n_tiles, int group_n, int last_width, int num_kb, int pairs) {
+    if (pairs <= 0 || pm_tiles <= 0 || n_tiles <= 0) return {0, 1, 0};
+    const int total = pm_tiles * n_tiles;
+    const int stagger = static_cast<int>(TAIL_EPI);
+    auto fits = [&](int ks) { return (num_kb - stagger * (ks * (ks - 1) / 2)) / ks >= TAIL_MIN_PART; };
+    // VPCE_TAIL_KS in the environment overrides the choice for A/B measurements: 0 = never split, k > 1 = the
+    // remainder tiles in k parts.
+    static const int forced = [] {
+        const char* e = getenv("VPCE_TAIL_KS");
+        return e ? atoi(e) : -1;
+    }();
+    if (forced == 0) return {0, 1, 0};
+    if (forced > 1) {
+        const int cut = std::min(std::min(total % pairs, total), MAX_SPLIT_TILES);
+        return (cut > 0 && fits(forced)) ? SplitChoice{cut, forced, stagger} : SplitChoice{0, 1, 0};
+    }
+    struct Key {
+        int a, b, c, d, e, f;
+        bool operator<(const Key& o) const { return std::tie(a, b, c, d, e, f) < std::tie(o.a, o.b, o.c, o.d, o.e, o.f); }
+    };
+    static std::mutex mu;
+    static std::map<Key, SplitChoice> cache;
+    const Key key{pm_tiles, n_tiles, group_n, last_width, num_kb, pairs};
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        auto it = cache.find(key);
+        if (it != cache.end()) return it->second;
+    }
+    const double c_last = last_width >= 256 ? 1.0 : std::max(0.875, last_width / 256.0);
+    SplitChoice best{0, 1, 0};
+    double best_t = simulate_tail(pm_tiles, n_tiles, group_n, c_last, 0, 1, 0, num_kb, pairs) * 0.98;   // a split must pay 2 %
+    const int R = total % pairs;
+    for (int cut : {R, R + pairs}) {
+        cut = std::min(std::min(cut, total), MAX_SPLIT_TILES);
+        if (cut <= 0) continue;
+        // two or three parts only: measured inside the power-capped benchmark step, more parts made the launch
+        // itself shorter but the step no faster (every part costs an epilogue and a pipeline fill of energy); a third
+        // part has to pay for itself
+        for (int ks : {2, 3}) {
+            if (!fits(ks)) break;
+            const double t = simulate_tail(pm_tiles, n_tiles, group_n, c_last, cut, ks, stagger, num_kb, pairs);
+            if (t < best_t) { best_t = t * (ks == 2 ? 0.985 : 1.0); best = {cut, ks, stagger}; }
+        }
+    }
+    std::lock_guard<std::mutex> lk(mu);
+    cache[key] = best;
+    return best;
 }
 
 // Which GEMMs run as CTA pairs (bit 0 strip kernels, bit 1 input-gradient, bit 2 weight-gradient).
@@ -394,6 +488,17 @@ cudaError_t fold_meeting(const FoldCtx& c, int x_row0, int rows, int w_row0, int
     return cudaGetLastError();
 }
 
+// Tail split of a gradient GEMM launched as CTA pairs (p.m_tiles, p.n_tiles, p.group_n, p.num_kb set; out_cols = N).
+void set_split(GemmParams& p, int64_t out_cols, CounterPool& counters, int width_unit = 128) {
+    const int left = static_cast<int>(out_cols - static_cast<int64_t>(p.n_tiles - 1) * 256);
+    const int last_width = left >= 256 ? 256 : (left + width_unit - 1) / width_unit * width_unit;
+    const SplitChoice c = pick_split((p.m_tiles + 1) / 2, p.n_tiles, p.group_n, last_width, p.num_kb, num_sms() / 2);
+    p.n_cut = c.n_cut;
+    p.k_split = c.ks;
+    p.k_stagger = c.stagger;
+    p.split_flags = c.n_cut > 0 ? counters.take_n(8 * c.n_cut) : nullptr;
+}
+
 // Tensor maps and workspace pointers of the backward meetings of one call.
 struct GradCtx {
     CUtensorMap tmX_k, tmW_k, tmW_khalf, tmG_st, tmG_k, tmW_mn, tmG_mn, tmX_mn, tmW_mn2, tmX_mn2;
@@ -499,7 +604,7 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         ph.c_row0 = 0; ph.accumulate = first ? 0 : 1;
         ph.status = c.status;
         ph.b_3d = c.mn3d;
-        ph.n_cut = pick_n_cut((ph.m_tiles + 1) / 2, ph.n_tiles, num_sms() / 2);
+        set_split(ph, d, counters);
         apply_tuning(ph, EPI_DH);
         ph.tile_counter = counters.take();
         if ((c.pmask & 2) && c.pair_ok && ph.m_tiles >= 2) e = launch_pair<256, false, true, EPI_DH>(c.tmG_k, c.tmW_mn2, tmAcc, ph, st);
@@ -529,7 +634,7 @@ cudaError_t grad_meeting(const GradCtx& c, int phases, int x_row0, int rows, int
         pw.c_row0 = 0; pw.accumulate = accumulate_dW ? 1 : 0;
         pw.status = c.status;
         pw.a_3d = c.mn3d; pw.b_3d = c.mn3d;
-        pw.n_cut = pick_n_cut((pw.m_tiles + 1) / 2, pw.n_tiles, num_sms() / 2);
+        set_split(pw, d, counters);
         apply_tuning(pw, EPI_DW);
         pw.tile_counter = counters.take();
         if ((c.pmask & 4) && c.pair_ok && pw.m_tiles >= 2) e = launch_pair<256, true, true, EPI_DW>(c.tmG_mn, c.tmX_mn2, tmDW, pw, st);

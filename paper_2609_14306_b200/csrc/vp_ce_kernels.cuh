@@ -27,7 +27,9 @@ struct GemmParams {
     int m_tiles, n_tiles, num_kb;
     int a_3d, b_3d;                        // MN-major operand fetched as one 3-D box (64 x 64 x chunks) per k-block
     int hint_a, hint_b, hint_c;            // L2 eviction hints for A loads, B loads, C stores: 0 normal, 1 first, 2 last
-    int n_cut;                             // pair kernel: full-width tiles run as two halves at the end of the list
+    int n_cut, k_split, k_stagger;         // pair kernel, gradient GEMMs: the last n_cut tiles of the list run as k_split parts along K,
+                                           // part j + 1 longer than part j by k_stagger k-blocks
+    int* split_flags;                      // [n_cut][8] zero before the launch: order of the parts' additions (see the pair kernel)
     int group_n;                           // n-tiles per raster group (tiles run m-major inside a group)
     int a_mn0, a_k0, b_mn0, b_k0;          // TMA coordinate bases (elements)
     int rows_valid;                        // valid accumulator rows overall (M bound)
@@ -606,17 +608,24 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         return left >= BN ? BN : ((left + R - 1) / R * R);
     };
     // The work list, handed out dynamically (greedy list scheduling):
-    //   [0, n_whole)                  256-row x BN tiles in raster order: n-fastest over ALL n-tiles of a row inside
-    //                                 raster groups, so the narrower last n-tile of a row runs next to the row's other
-    //                                 tiles and shares their A rows through L2 (placing those tiles at the end of the
-    //                                 list re-read the whole A operand from DRAM);
-    //   [n_whole, n_whole + 2*n_cut)  the last n_cut tiles as two 128-column halves each (gradient GEMMs only, and only
-    //                                 when the host's estimate says the last round ends sooner that way).
+    //   [0, n_whole)                      256-row x BN tiles in raster order: n-fastest over ALL n-tiles of a row inside
+    //                                     raster groups, so the narrower last n-tile of a row runs next to the row's other
+    //                                     tiles and shares their A rows through L2;
+    //   [n_whole, n_whole + ks * n_cut)   the last n_cut tiles as ks parts each along K (gradient GEMMs only; the host
+    //                                     picks n_cut and ks so that the last round of the list ends sooner).  Part j + 1
+    //                                     is k_stagger k-blocks longer than part j: parts taken together then finish one
+    //                                     after the other, an epilogue apart, instead of queueing.  The parts of a tile add
+    //                                     into the same output elements, in the order of j: each epilogue warp waits for
+    //                                     the warp that wrote the same rows of part j - 1 (a flag in global memory), so the
+    //                                     fp32 sum has one fixed order whatever pairs ran the parts.  A part is always taken
+    //                                     from the list after the parts it waits for, and those never wait for a later
+    //                                     entry, so the waits cannot form a cycle.
     constexpr bool kSplit = (EPI == EPI_DH || EPI == EPI_DW);
     const int total_tiles = pm_tiles * p.n_tiles;
     const int n_cut = kSplit ? min(p.n_cut, total_tiles) : 0;
+    const int ks = n_cut > 0 ? max(p.k_split, 1) : 1;
     const int n_whole = total_tiles - n_cut;
-    const int list_len = n_whole + 2 * n_cut;
+    const int list_len = n_whole + ks * n_cut;
     auto decode_raster = [&](int tile, int& pmt, int& nt) {
         const int per_group = p.group_n * pm_tiles;
         const int g = tile / per_group;
@@ -626,18 +635,28 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         pmt = r / gw;
         nt = n0 + (r - pmt * gw);
     };
-    // Entry t of the list: 256-row tile pmt, columns [ncol0, ncol0 + width) of n-tile nt; width == 0 means "nothing".
-    auto get_tile = [&](int t, int& pmt, int& nt, int& ncol0, int& width) {
+    // Entry t of the list: 256-row tile pmt, n-tile nt (columns [ncol0, ncol0 + width)), k-blocks [kb0, kb1);
+    // part j of split tile number `slot` (slot < 0: a whole tile).
+    struct Work { int pmt, nt, ncol0, width, kb0, kb1, part, slot; };
+    auto get_tile = [&](int t) {
+        Work w;
         if (t < n_whole) {
-            decode_raster(t, pmt, nt);
-            ncol0 = nt * BN; width = tile_n(nt);
-            return;
+            decode_raster(t, w.pmt, w.nt);
+            w.kb0 = 0; w.kb1 = p.num_kb; w.part = 0; w.slot = -1;
+        } else {
+            const int v = t - n_whole;
+            w.slot = v / ks;
+            w.part = v - w.slot * ks;
+            decode_raster(n_whole + w.slot, w.pmt, w.nt);
+            // part lengths base, base + dk, base + 2 dk, ...; the last part also takes what the division leaves
+            const int dk = p.k_stagger;
+            const int base_len = (p.num_kb - dk * (ks * (ks - 1) / 2)) / ks;
+            w.kb0 = w.part * base_len + dk * (w.part * (w.part - 1) / 2);
+            w.kb1 = w.part + 1 == ks ? p.num_kb : w.kb0 + base_len + dk * w.part;
         }
-        const int v = t - n_whole;
-        decode_raster(n_whole + (v >> 1), pmt, nt);
-        const int w = tile_n(nt);
-        if (w <= BN / 2) { ncol0 = nt * BN; width = (v & 1) ? 0 : w; }
-        else { ncol0 = nt * BN + (v & 1) * (BN / 2); width = (v & 1) ? w - BN / 2 : BN / 2; }
+        w.ncol0 = w.nt * BN;
+        w.width = tile_n(w.nt);
+        return w;
     };
     // Scheduler ring: the leader's producer lane takes list positions from the launch's counter and writes them
     // into the same slot of both CTAs; every reader acknowledges on the leader's "slot free" barrier.
@@ -679,18 +698,16 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
                 }
                 if (tile < 0) break;
-                int pmt, nt, ncol0, width;
-                get_tile(tile, pmt, nt, ncol0, width);
-                if (width == 0) continue;
-                const int mt = 2 * pmt + static_cast<int>(rank);             // this CTA's 128-row tile
-                const int bn0 = ncol0 + static_cast<int>(rank) * (width / 2);   // this CTA's half of the B tile
-                for (int kb = 0; kb < p.num_kb; ++kb) {
+                const Work w = get_tile(tile);
+                const int mt = 2 * w.pmt + static_cast<int>(rank);           // this CTA's 128-row tile
+                const int bn0 = w.ncol0 + static_cast<int>(rank) * (w.width / 2);   // this CTA's half of the B tile
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
                     const uint32_t bar = mapa_shared(full_bar(stage), 0);    // the leader's barrier
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
                     const uint32_t sb = sa + Cfg::A_BYTES;
-                    const bool drop = tile == 0 && kb == p.drop_kb && ((p.drop_ranks >> rank) & 1);   // test hook
+                    const bool drop = tile == 0 && kb - w.kb0 == p.drop_kb && ((p.drop_ranks >> rank) & 1);   // test hook
                     if (!drop) {
                         if (A_MN) tma2_load_3d(sa, &tmA, bar, 0, p.a_k0 + kb * BKE, (p.a_mn0 + mt * BM) >> CSH, pol_a);
                         else tma2_load_2d(sa, &tmA, bar, p.a_k0 + kb * BKE, p.a_mn0 + mt * BM, pol_a);
@@ -723,16 +740,14 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 sched_ack(ss);
                 if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
                 if (tile < 0) break;
-                int pmt, nt, ncol0, width;
-                get_tile(tile, pmt, nt, ncol0, width);
-                if (width == 0) continue;
-                const uint32_t idesc = make_idesc(width, A_MN, B_MN, 2 * BM, TF32 ? 2u : 1u);
+                const Work w = get_tile(tile);
+                const uint32_t idesc = make_idesc(w.width, A_MN, B_MN, 2 * BM, TF32 ? 2u : 1u);
                 const int ab = it & 1;
                 const uint32_t aphase = (it >> 1) & 1u;
                 if (!mbar_wait_cluster(tempty_bar(ab), aphase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + ab * ACC_STRIDE;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
@@ -747,8 +762,8 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         // K-major: UK elements = 32 B along the swizzled row; MN-major: UK k-rows of 128 B
                         const uint64_t aoff = static_cast<uint64_t>((A_MN ? k * UK * 128 : k * 32) >> 4);
                         const uint64_t boff = static_cast<uint64_t>((B_MN ? k * UK * 128 : k * 32) >> 4);
-                        if (TF32) umma2_tf32(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
-                        else umma2_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb | k) != 0 ? 1u : 0u);
+                        if (TF32) umma2_tf32(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb > w.kb0 || k != 0) ? 1u : 0u);
+                        else umma2_f16(tmem_d, adesc + aoff, bdesc + boff, idesc, (kb > w.kb0 || k != 0) ? 1u : 0u);
                     }
                     umma2_commit_both(empty_bar(stage));                     // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -779,10 +794,9 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             tile = __shfl_sync(0xffffffffu, tile, 0);
             if (++ss == SCHED_DEPTH) { ss = 0; sphase ^= 1u; }
             if (tile < 0) break;                                             // -1: list exhausted, -2: gave up
-            int pmt, nt, ncol0, width;
-            get_tile(tile, pmt, nt, ncol0, width);
-            if (width == 0) continue;
-            const int mt = 2 * pmt + static_cast<int>(rank);
+            const Work w = get_tile(tile);
+            const int mt = 2 * w.pmt + static_cast<int>(rank);
+            const int nt = w.nt;
             const int ab = it & 1;
             const uint32_t aphase = (it >> 1) & 1u;
             if (!mbar_wait(tfull_bar(ab), aphase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
@@ -791,8 +805,20 @@ vpce_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (EPI == EPI_FOLD) epilogue_fold(p, mt, nt, row, tmem_row);
             else if (EPI == EPI_RESID && TF32) epilogue_resid_f32(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
             else if (EPI == EPI_RESID) epilogue_resid(p, &tmC, g_staging + (warp - 2) * 8192, mt, nt, row, lane, tmem_row);
-            else epilogue_f32_tile(&tmC, g_staging + (warp - 2) * 8192, ncol0, p.c_row0 + mt * BM + quad * 32, lane, tmem_row,
-                                   width, p.accumulate != 0);
+            else {
+                // parts of a split tile add in the order of their index: wait for this warp's rows of the part before
+                int* flag = w.slot >= 0 ? p.split_flags + w.slot * 8 + static_cast<int>(rank) * 4 + quad : nullptr;
+                if (w.part > 0) {
+                    if (lane == 0 && !flag_wait_ge(flag, w.part, abort_flag, p.wait_limit_ns)) ok = false;
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                }
+                epilogue_f32_tile(&tmC, g_staging + (warp - 2) * 8192, w.ncol0, p.c_row0 + mt * BM + quad * 32, lane, tmem_row,
+                                  w.width, p.accumulate != 0 || w.part > 0);
+                if (flag != nullptr && w.part + 1 < ks && lane == 0) {
+                    bulk_wait_all();                                         // this warp's stores / additions are complete
+                    flag_release(flag, w.part + 1);
+                }
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(ab), 0));   // the leader owns this barrier
