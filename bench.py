@@ -37,10 +37,10 @@ FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_g
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel kind, from ncu captures of
 # launches of the same geometry, keyed by (dtype, d, block_v, T_chunk); other geometries report traffic = null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("bf16", 2880, 8192, 16384): {"fwd_strip_fold": 156e6, "bwd_strip_residual": 462e6, "dH_gemm": 882e6,
-                                  "dW_gemm": 972e6},
-    ("bf16", 7168, 8192, 8192): {"fwd_strip_fold": 596e6, "bwd_strip_residual": 782e6, "dH_gemm": 1073e6,
-                                 "dW_gemm": 1076e6},
+    ("bf16", 2880, 8192, 16384): {"fwd_strip_fold": 159e6, "bwd_strip_residual": 484e6, "dH_gemm": 926e6,
+                                  "dW_gemm": 969e6},
+    ("bf16", 7168, 8192, 8192): {"fwd_strip_fold": 692e6, "bwd_strip_residual": 898e6, "dH_gemm": 1147e6,
+                                 "dW_gemm": 1141e6},
 }
 # Token chunk used by the timed launch configuration (a call argument of the library).
 BENCH_T_CHUNK = {"tiny": 512, "mid": 4096, "moe120b": 16384, "moe667b": 8192, "longctx": 16384}
