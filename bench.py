@@ -623,6 +623,8 @@ def main():
                     help="skip the extra measured blocks (the other target configuration, the paper's shape in TF32)")
     ap.add_argument("--no-yardstick", action="store_true", help="skip the cuBLAS context measurement")
     ap.add_argument("--profile-in-timed-region", type=int, default=1)
+    ap.add_argument("--tail-parts", type=int, default=-1,
+                    help="A/B knob of the gradient GEMMs' K-split tail (vp_ce_set_tail_parts): -1 library's choice, 0 off")
     ap.add_argument("--adamw", default="", help="measure only the streamed AdamW: parameters,bucket,slots (e.g. 268435456,100000000,2)")
     args = ap.parse_args()
 
@@ -644,6 +646,8 @@ def main():
     import paper_2609_14306_b200 as vp
     ctx = Ctx()
     vp.load_library()          # raises if the CUDA library is missing: there is no fallback
+    if args.tail_parts != -1:
+        vp.vp_ce_set_tail_parts(args.tail_parts)
 
     if args.adamw:
         n_, b_, s_ = (int(x) for x in args.adamw.split(","))

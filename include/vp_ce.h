@@ -258,6 +258,19 @@ vpce_status vp_ce_backward_f32(const float* H, const float* W, const int32_t* la
 int64_t vp_ce_set_wait_limit_ns(int64_t ns);
 
 /*
+ * Tuning knob (no counterpart in the paper).  When the 256 x 256 output tiles of a gradient GEMM
+ * do not fill a whole number of rounds of the CTA pairs, the remainder tiles are run as two or
+ * three parts along the contracted dimension; the parts of a tile add into the output in the order
+ * of their index (flags in the workspace), so results stay bitwise reproducible for a given
+ * setting.  vp_ce_set_tail_parts(parts) overrides the library's choice for all later launches of
+ * this process: -1 = the library decides per launch geometry (default), 0 = never split,
+ * 2..8 = the remainder tiles in that many parts whenever the contraction is long enough.  Other
+ * values change nothing.  Returns the previous setting.  Results of different settings differ in
+ * the last bits (another summation order).
+ */
+int vp_ce_set_tail_parts(int parts);
+
+/*
  * TEST HOOK (no counterpart in the paper): makes one copy of the next launch "get lost" so that
  * the give-up path above can be exercised without any invalid access.  The next launch of kernel
  * kind `kernel_kind` (0 forward strip, 1 backward strip, 2 input-gradient GEMM, 3 weight-gradient

@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     vp_ce_fwd_bwd_host,
     vp_ce_profile_collect,
     vp_ce_profile_enable,
+    vp_ce_set_tail_parts,
     vp_ce_set_wait_limit_ns,
     vp_ce_debug_drop_copy,
     KERNEL_KINDS,

@@ -81,6 +81,8 @@ def load_library() -> ctypes.CDLL:
                                        ctypes.c_int, vp, sz, vp]
     lib.vp_ce_set_wait_limit_ns.restype = i64
     lib.vp_ce_set_wait_limit_ns.argtypes = [i64]
+    lib.vp_ce_set_tail_parts.restype = ctypes.c_int
+    lib.vp_ce_set_tail_parts.argtypes = [ctypes.c_int]
     lib.vp_ce_debug_drop_copy.restype = ctypes.c_int
     lib.vp_ce_debug_drop_copy.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
     f32 = ctypes.c_float
@@ -308,6 +310,12 @@ def vp_ce_fwd_bwd_host(H_host, labels_host, W, loss_host, dH_host, dW, block_v: 
 def vp_ce_set_wait_limit_ns(ns: int) -> int:
     """Sets the limit of every wait inside the kernels (ns <= 0: query only); returns the previous limit."""
     return int(load_library().vp_ce_set_wait_limit_ns(int(ns)))
+
+
+def vp_ce_set_tail_parts(parts: int) -> int:
+    """Overrides how the remainder tiles of the gradient GEMMs are split along K (-1 library's choice, 0 never,
+    2..8 that many parts); returns the previous setting."""
+    return int(load_library().vp_ce_set_tail_parts(int(parts)))
 
 
 def vp_ce_debug_drop_copy(kernel_kind: int, k_block: int = 0, cta_ranks: int = 1) -> None:

@@ -64,6 +64,8 @@ std::vector<ProfEntry> g_prof;
 // in bits 24-27; -1 = nothing armed.
 std::atomic<unsigned long long> g_wait_limit_ns{kDefaultWaitLimitNs};
 std::atomic<int> g_drop{-1};
+// vp_ce_set_tail_parts: -1 the host decides, 0 never split, k > 1 the remainder tiles in k parts.
+std::atomic<int> g_tail_parts{-1};
 
 // Fills the launch-time fields every GEMM launch shares.
 GemmParams finish_params(const GemmParams& p, int epi) {
@@ -328,16 +330,12 @@ SplitChoice pick_split(int pm_tiles, int n_tiles, int group_n, int last_width, i
     const int total = pm_tiles * n_tiles;
     const int stagger = static_cast<int>(TAIL_EPI);
     auto fits = [&](int ks) { return (num_kb - stagger * (ks * (ks - 1) / 2)) / ks >= TAIL_MIN_PART; };
-    // VPCE_TAIL_KS in the environment overrides the choice for A/B measurements: 0 = never split, k > 1 = the
-    // remainder tiles in k parts.
-    static const int forced = [] {
-        const char* e = getenv("VPCE_TAIL_KS");
-        return e ? atoi(e) : -1;
-    }();
+    const int forced = g_tail_parts.load(std::memory_order_relaxed);          // vp_ce_set_tail_parts overrides the choice
     if (forced == 0) return {0, 1, 0};
-    if (forced > 1) {
+    if (forced > 1) {                      // as asked, staggered when K is long enough for it, else in equal parts
         const int cut = std::min(std::min(total % pairs, total), MAX_SPLIT_TILES);
-        return (cut > 0 && fits(forced)) ? SplitChoice{cut, forced, stagger} : SplitChoice{0, 1, 0};
+        if (cut <= 0 || num_kb < forced) return {0, 1, 0};
+        return fits(forced) ? SplitChoice{cut, forced, stagger} : SplitChoice{cut, forced, 0};
     }
     struct Key {
         int a, b, c, d, e, f;
@@ -930,6 +928,12 @@ int64_t vp_ce_set_wait_limit_ns(int64_t ns) {
         g_wait_limit_ns.store(v, std::memory_order_relaxed);
     }
     return static_cast<int64_t>(prev);
+}
+
+int vp_ce_set_tail_parts(int parts) {
+    const int prev = g_tail_parts.load(std::memory_order_relaxed);
+    if (parts >= -1 && parts != 1 && parts <= 8) g_tail_parts.store(parts, std::memory_order_relaxed);
+    return prev;
 }
 
 vpce_status vp_ce_debug_drop_copy(int kernel_kind, int k_block, int cta_ranks) {

@@ -69,6 +69,11 @@ def test_wait_limit_and_test_hook_arguments():
             vp.vp_ce_debug_drop_copy(*bad)
     vp.vp_ce_debug_drop_copy(2, 3, 3)
     vp.vp_ce_debug_drop_copy(-1)                              # disarm
+    # the tail-split knob: -1 (library's choice) by default; 1, 9 and -2 are ignored
+    assert vp.vp_ce_set_tail_parts(3) == -1
+    assert vp.vp_ce_set_tail_parts(1) == 3 and vp.vp_ce_set_tail_parts(9) == 3 and vp.vp_ce_set_tail_parts(-2) == 3
+    assert vp.vp_ce_set_tail_parts(0) == 3
+    assert vp.vp_ce_set_tail_parts(-1) == 0
 
 
 def test_streamed_adamw_staging_size():
