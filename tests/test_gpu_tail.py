@@ -60,6 +60,29 @@ def test_forced_split_matches_oracle_and_is_reproducible(tail_parts, parts, T, d
     assert (a.dW != whole.dW).any(), "the split did not change the summation order: was it applied at all?"
 
 
+@pytest.mark.parametrize("parts", [-1, 3])
+def test_split_tail_is_bitwise_reproducible_at_the_benchmark_launch_geometry(tail_parts, parts):
+    # the config-3 launch geometry (74 pairs, 384 / 768 tiles per gradient launch, 14 / 28 remainder tiles, narrow
+    # last column tile), two shards; -1 is the library's own choice, which splits the weight-gradient launch here
+    w = custom_workload("tailrep", T=16384, d=2880, V=16384, block_v=8192, T_chunk=16384, w_std=0.02,
+                        labels="zipf", ignore_frac=0.05, seed=9)
+    b = make_batch(w)
+    tail_parts(0)
+    whole = _run(w, b, base=1)
+    tail_parts(parts)
+    run = _run(w, b, base=1)
+    assert run.bwd_status == 0
+    dW0, dH0 = run.dW.clone(), run.dH.clone()
+    assert (dW0 != whole.dW).any()                            # the split is in use
+    assert relF(dW0.double().cpu().numpy(), whole.dW.double().cpu().numpy()) <= 1e-5
+    for _ in range(10):
+        run.dW.fill_(float("nan"))
+        run.dH.fill_(float("nan"))
+        run.backward()
+        assert run.bwd_status == 0
+        assert torch.equal(run.dW, dW0) and torch.equal(run.dH.view(torch.int16), dH0.view(torch.int16))
+
+
 def test_lost_copy_inside_a_split_tile_gives_up_and_the_next_call_is_clean(tail_parts):
     w = custom_workload("tailgiveup", T=512, d=256, V=1024, block_v=512, T_chunk=256, w_std=0.0625,
                         labels="zipf", ignore_frac=0.05, seed=62)
