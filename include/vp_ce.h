@@ -271,6 +271,18 @@ int64_t vp_ce_set_wait_limit_ns(int64_t ns);
 int vp_ce_set_tail_parts(int parts);
 
 /*
+ * The decision the library takes for a gradient GEMM of the given launch geometry (pure host
+ * arithmetic, no device needed): row_tiles x col_tiles output tiles of 256 x 256 handed out to
+ * `pairs` CTA pairs in raster groups of group_cols column tiles, the last column tile with an MMA
+ * width of last_width (<= 256), k_blocks k-blocks (of 64 bf16 / 32 fp32 elements) in the
+ * contraction.  Outputs: how many tiles at the end of the work list are split, into how many
+ * parts, and by how many k-blocks each part is longer than the one before it (0 tiles = no
+ * split).  Honours vp_ce_set_tail_parts.  Returns VPCE_INVALID_ARG for non-positive arguments.
+ */
+vpce_status vp_ce_tail_choice(int row_tiles, int col_tiles, int group_cols, int last_width, int k_blocks, int pairs,
+                              int* n_tiles_split, int* parts, int* stagger);
+
+/*
  * TEST HOOK (no counterpart in the paper): makes one copy of the next launch "get lost" so that
  * the give-up path above can be exercised without any invalid access.  The next launch of kernel
  * kind `kernel_kind` (0 forward strip, 1 backward strip, 2 input-gradient GEMM, 3 weight-gradient

@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     vp_ce_profile_collect,
     vp_ce_profile_enable,
     vp_ce_set_tail_parts,
+    vp_ce_tail_choice,
     vp_ce_set_wait_limit_ns,
     vp_ce_debug_drop_copy,
     KERNEL_KINDS,

@@ -83,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.vp_ce_set_wait_limit_ns.argtypes = [i64]
     lib.vp_ce_set_tail_parts.restype = ctypes.c_int
     lib.vp_ce_set_tail_parts.argtypes = [ctypes.c_int]
+    lib.vp_ce_tail_choice.restype = ctypes.c_int
+    lib.vp_ce_tail_choice.argtypes = [ctypes.c_int] * 6 + [ctypes.POINTER(ctypes.c_int)] * 3
     lib.vp_ce_debug_drop_copy.restype = ctypes.c_int
     lib.vp_ce_debug_drop_copy.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
     f32 = ctypes.c_float
@@ -316,6 +318,14 @@ def vp_ce_set_tail_parts(parts: int) -> int:
     """Overrides how the remainder tiles of the gradient GEMMs are split along K (-1 library's choice, 0 never,
     2..8 that many parts); returns the previous setting."""
     return int(load_library().vp_ce_set_tail_parts(int(parts)))
+
+
+def vp_ce_tail_choice(row_tiles: int, col_tiles: int, group_cols: int, last_width: int, k_blocks: int, pairs: int):
+    """(tiles split, parts, stagger) the library picks for a gradient GEMM of that launch geometry (host only)."""
+    n, k, s = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    _check(load_library().vp_ce_tail_choice(int(row_tiles), int(col_tiles), int(group_cols), int(last_width),
+                                            int(k_blocks), int(pairs), ctypes.byref(n), ctypes.byref(k), ctypes.byref(s)))
+    return n.value, k.value, s.value
 
 
 def vp_ce_debug_drop_copy(kernel_kind: int, k_block: int = 0, cta_ranks: int = 1) -> None:

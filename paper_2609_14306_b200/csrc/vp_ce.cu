@@ -936,6 +936,18 @@ int vp_ce_set_tail_parts(int parts) {
     return prev;
 }
 
+vpce_status vp_ce_tail_choice(int row_tiles, int col_tiles, int group_cols, int last_width, int k_blocks, int pairs,
+                              int* n_tiles_split, int* parts, int* stagger) {
+    if (row_tiles <= 0 || col_tiles <= 0 || group_cols <= 0 || last_width <= 0 || last_width > 256 || k_blocks <= 0 ||
+        pairs <= 0 || !n_tiles_split || !parts || !stagger)
+        return VPCE_INVALID_ARG;
+    const SplitChoice c = pick_split(row_tiles, col_tiles, group_cols, last_width, k_blocks, pairs);
+    *n_tiles_split = c.n_cut;
+    *parts = c.ks;
+    *stagger = c.stagger;
+    return VPCE_OK;
+}
+
 vpce_status vp_ce_debug_drop_copy(int kernel_kind, int k_block, int cta_ranks) {
     if (kernel_kind < 0) { g_drop.store(-1, std::memory_order_relaxed); return VPCE_OK; }
     if (kernel_kind > 3 || k_block < 0 || k_block > 0xffff || cta_ranks <= 0 || cta_ranks > 3) return VPCE_INVALID_ARG;

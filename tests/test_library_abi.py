@@ -81,3 +81,40 @@ def test_streamed_adamw_staging_size():
     assert vp.osadamw_staging_bytes(1 << 20, 2) == 2 * 4 * (1 << 20) * 4
     assert vp.osadamw_staging_bytes(100, 3) == 3 * 4 * 128 * 4
     assert vp.osadamw_staging_bytes(0, 2) == 0 and vp.osadamw_staging_bytes(100, 0) == 0
+
+
+def test_tail_choice_of_the_gradient_gemms():
+    """Host logic of the K-split tail: which remainder tiles are split, into how many parts."""
+    import pytest
+    assert vp.vp_ce_set_tail_parts(-1) == -1
+    # config 3, weight gradient: 32 x 12 tiles (last column tile 128 wide in the MMA), 2 raster groups, K = 16384 tokens:
+    # 384 % 74 = 14 remainder tiles, split (the launch measured 6 % shorter that way)
+    n, parts, stagger = vp.vp_ce_tail_choice(32, 12, 6, 128, 256, 74)
+    assert n == 14 and parts in (2, 3) and stagger == 15
+    # config 4: 32 x 28 whole tiles, K = 8192: 896 % 74 = 8 remainder tiles
+    n, parts, stagger = vp.vp_ce_tail_choice(32, 28, 7, 256, 128, 74)
+    assert n == 8 and parts in (2, 3)
+    # a whole number of rounds: nothing to split
+    assert vp.vp_ce_tail_choice(37, 10, 10, 256, 256, 74) == (0, 1, 0)
+    # almost a full last round (70 of 74 pairs busy): a split cannot pay
+    assert vp.vp_ce_tail_choice(36, 4, 4, 256, 256, 74)[0] == 0
+    # a contraction too short for two parts of 8 k-blocks plus the stagger: no split
+    assert vp.vp_ce_tail_choice(8, 10, 10, 256, 24, 74) == (0, 1, 0)
+    # the knob: 0 forbids, k forces (equal parts when K is too short for staggered ones)
+    vp.vp_ce_set_tail_parts(0)
+    try:
+        assert vp.vp_ce_tail_choice(32, 12, 6, 128, 256, 74) == (0, 1, 0)
+        vp.vp_ce_set_tail_parts(4)
+        assert vp.vp_ce_tail_choice(32, 12, 6, 128, 256, 74) == (14, 4, 15)
+        assert vp.vp_ce_tail_choice(4, 2, 2, 128, 16, 74) == (8, 4, 0)
+        assert vp.vp_ce_tail_choice(4, 2, 2, 128, 3, 74) == (0, 1, 0)       # fewer k-blocks than parts
+    finally:
+        vp.vp_ce_set_tail_parts(-1)
+    # never more split tiles than flags in the workspace allow, never more parts than three by the library's own choice
+    for rows, cols, kb in [(64, 12, 128), (98, 28, 256), (16, 8, 32), (5, 3, 512), (1, 1, 64), (64, 28, 392)]:
+        n, parts, stagger = vp.vp_ce_tail_choice(rows, cols, min(cols, 7), 256, kb, 74)
+        assert 0 <= n <= 64 and 1 <= parts <= 3 and (n == 0) == (parts == 1)
+        if n:
+            assert (kb - stagger * parts * (parts - 1) // 2) // parts >= 8
+    with pytest.raises(vp.VpceError):
+        vp.vp_ce_tail_choice(0, 1, 1, 256, 64, 74)
