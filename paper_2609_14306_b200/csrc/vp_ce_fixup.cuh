@@ -110,12 +110,12 @@ vpce_finish_dx_kernel(float* __restrict__ acc, __nv_bfloat16* __restrict__ out, 
     }
 }
 
-// First position of the sorted keys[0, n) whose key is >= x, found by all 256 threads of the CTA together: two rounds of
+// First position of the sorted keys[0, n) whose key is >= x, found by all 256 threads of the CTA together: two steps of
 // parallel probes (every 64th key, then the 64 keys of the bracket) instead of a 14-step dependent chain.
 __device__ __forceinline__ int block_lower_bound(const unsigned long long* keys, int n, unsigned long long x, int* s_tmp) {
     if (threadIdx.x == 0) *s_tmp = n;
     __syncthreads();
-    // round 1: the first probe position p = 64 k (k = 0 .. 255, + tail) with keys[p] >= x
+    // step 1: the first probe position p = 64 k (k = 0 .. 255, + tail) with keys[p] >= x
     for (int p = threadIdx.x * 64; p < n; p += 256 * 64)
         if (keys[p] >= x) atomicMin(s_tmp, p);
     __syncthreads();
